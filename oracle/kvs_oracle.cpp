@@ -1,0 +1,439 @@
+// CPU oracle for the KV-memory-constrained schedule builder and evaluator.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, single-threaded, literal
+// restatement of the paper's definitions that the CUDA library is checked
+// against.  It shares no code with the CUDA path and must never be linked,
+// imported or called from it; only the tests, the smoke check and the CPU
+// baseline leg of the benchmark use it.
+//
+// What each part follows (paper passages):
+//   * memory of an active job and feasibility        - Preliminaries, Eq. (Memory-Feasibility)
+//   * total flow time                                 - Preliminaries, "Objective and Benchmark"
+//   * Staggered-Pipeline-Schedule (SPS)               - Procedure "StaggeredPipelineSchedule"
+//   * Peak(k, tau, s) and k*(tau, s)                  - Lemma "Peak Memory Usage of SPS",
+//                                                       Lemma "Feasible Parallelism of SPS", Eq. (max-parallelism)
+//   * Geometric-Slicing-Algorithm (GSA)               - Algorithm "Geometric Slicing Algorithm"
+//   * Geometric-Batching-Algorithm (GBA)              - Algorithm "Geometric Batching Algorithm"
+//   * Simultaneous-Schedule (SimS)                    - Appendix "Lower Bounds for SimS", batch size B
+//   * optimum without kills or pauses (brute force)   - footnote to the definition of competitive ratio
+//
+// Parity status.  Pinned by the paper: SPS, SimS, Peak, k*, GBA and GSA with
+// exact response lengths, the dense evaluator (Example 1 memory columns, flow
+// 180 / 225; uniform experiment 14083 and 21632; long-job-trap closed form;
+// two-point experiment range).  PARITY UNPINNED (no counterpart in the paper,
+// pinned only by reductions to the paper's cases and by invariants):
+//   * schedules built on estimates (class by estimate, kill-and-carry),
+//   * arrival windows,
+//   * heterogeneous prompt lengths (one scalar s_bar for ladder and k*).
+//
+// All quantities are exact integers (int64); nothing here is floating point.
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+typedef int64_t i64;
+typedef uint64_t u64;
+
+// ---------------------------------------------------------------------------
+// Minimal unsigned big integer (little-endian 32-bit limbs): only what the
+// exact ladder needs - multiply by a small number, multiply by a 64-bit number,
+// compare.
+// ---------------------------------------------------------------------------
+struct Big {
+  std::vector<uint32_t> limb;
+  explicit Big(u64 v = 0) {
+    while (v) { limb.push_back(static_cast<uint32_t>(v)); v >>= 32; }
+  }
+  void mul_small(uint32_t m) {
+    u64 carry = 0;
+    for (size_t i = 0; i < limb.size(); ++i) {
+      u64 cur = static_cast<u64>(limb[i]) * m + carry;
+      limb[i] = static_cast<uint32_t>(cur);
+      carry = cur >> 32;
+    }
+    if (carry) limb.push_back(static_cast<uint32_t>(carry));
+    trim();
+  }
+  void trim() { while (!limb.empty() && limb.back() == 0) limb.pop_back(); }
+  Big times_u64(u64 m) const {
+    Big lo = *this, hi = *this;
+    lo.mul_small(static_cast<uint32_t>(m));
+    hi.mul_small(static_cast<uint32_t>(m >> 32));
+    // result = lo + (hi << 32)
+    Big r;
+    r.limb.assign(std::max(lo.limb.size(), hi.limb.size() + 1) + 1, 0);
+    u64 carry = 0;
+    for (size_t i = 0; i < r.limb.size(); ++i) {
+      u64 cur = carry;
+      if (i < lo.limb.size()) cur += lo.limb[i];
+      if (i >= 1 && i - 1 < hi.limb.size()) cur += hi.limb[i - 1];
+      r.limb[i] = static_cast<uint32_t>(cur);
+      carry = cur >> 32;
+    }
+    r.trim();
+    return r;
+  }
+  // -1, 0, +1
+  static int cmp(const Big& x, const Big& y) {
+    if (x.limb.size() != y.limb.size()) return x.limb.size() < y.limb.size() ? -1 : 1;
+    for (size_t i = x.limb.size(); i-- > 0;)
+      if (x.limb[i] != y.limb[i]) return x.limb[i] < y.limb[i] ? -1 : 1;
+    return 0;
+  }
+};
+
+Big big_pow(uint32_t base, int e) {
+  Big r(1);
+  for (int i = 0; i < e; ++i) r.mul_small(base);
+  return r;
+}
+
+// floor(X * b^j / a^j) for alpha = a/b > 1: the largest integer t with t * a^j <= X * b^j.
+i64 floor_scaled(i64 X, int a, int b, int j) {
+  Big rhs = big_pow(static_cast<uint32_t>(b), j).times_u64(static_cast<u64>(X));
+  Big aj = big_pow(static_cast<uint32_t>(a), j);
+  i64 lo = 0, hi = X;  // alpha > 1 so the answer is in [0, X]
+  while (lo < hi) {
+    i64 mid = lo + (hi - lo + 1) / 2;
+    if (Big::cmp(aj.times_u64(static_cast<u64>(mid)), rhs) <= 0) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+i64 gcd64(i64 x, i64 y) { while (y) { i64 t = x % y; x = y; y = t; } return x; }
+
+// Peak(k, tau, s) = s*k + (tau*k + tau + k - gcd(tau, k)) / 2   (peak-memory lemma)
+i64 peak_closed(i64 k, i64 tau, i64 s) {
+  return s * k + (tau * k + tau + k - gcd64(tau, k)) / 2;
+}
+
+// k*(tau, s) = max{k >= 1 : Peak(k, tau, s) <= M}  (Eq. max-parallelism); 0 if even k = 1 does
+// not fit.  Peak is increasing in k (same lemma), so a doubling + bisection search is exact.
+i64 kstar(i64 tau, i64 s, i64 M) {
+  if (peak_closed(1, tau, s) > M) return 0;
+  i64 lo = 1, hi = 2;
+  while (peak_closed(hi, tau, s) <= M) { lo = hi; hi *= 2; }
+  while (hi - lo > 1) {
+    i64 mid = lo + (hi - lo) / 2;
+    if (peak_closed(mid, tau, s) <= M) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// Geometric ladder of integer slice lengths tau_0 .. tau_ell.
+//   paper's initialisation (beta0 == 0): ell = floor(log_alpha X), tau_hat_0 = X / alpha^ell,
+//     tau_p = floor(tau_hat_0 * alpha^p) = floor(X / alpha^(ell-p)), so tau_ell = X exactly;
+//   tunable initial slice (beta0 > 0): tau_p = min(floor(beta0 * alpha^p), X), last phase is the
+//     first one that reaches X.
+std::vector<i64> ladder(i64 X, int a, int b, i64 beta0) {
+  std::vector<i64> tau;
+  if (X < 1 || a <= b || b < 1) return tau;
+  if (beta0 <= 0) {
+    int ell = 0;  // largest j with a^j <= X * b^j
+    while (Big::cmp(big_pow(static_cast<uint32_t>(a), ell + 1),
+                    big_pow(static_cast<uint32_t>(b), ell + 1).times_u64(static_cast<u64>(X))) <= 0)
+      ++ell;
+    for (int p = 0; p <= ell; ++p) tau.push_back(floor_scaled(X, a, b, ell - p));
+  } else {
+    for (int p = 0;; ++p) {
+      // floor(beta0 * a^p / b^p): largest t with t * b^p <= beta0 * a^p, capped at X.
+      Big rhs = big_pow(static_cast<uint32_t>(a), p).times_u64(static_cast<u64>(beta0));
+      Big bp = big_pow(static_cast<uint32_t>(b), p);
+      i64 t;
+      if (Big::cmp(bp.times_u64(static_cast<u64>(X)), rhs) <= 0) {
+        t = X;
+      } else {
+        i64 lo = 0, hi = X;
+        while (lo < hi) {
+          i64 mid = lo + (hi - lo + 1) / 2;
+          if (Big::cmp(bp.times_u64(static_cast<u64>(mid)), rhs) <= 0) lo = mid; else hi = mid - 1;
+        }
+        t = lo;
+      }
+      tau.push_back(t);
+      if (t >= X) break;
+    }
+  }
+  return tau;
+}
+
+enum { FAM_GBA = 0, FAM_GSA = 1, FAM_SPS = 2, FAM_SIMS = 3 };
+
+struct Run { i64 job, phase, start, len, s; };
+
+struct Schedule {
+  int status = 0;               // 0 ok, 1 a job (or the slice) cannot fit, 3 bad arguments
+  i64 n = 0;
+  i64 s_bar = 0;
+  std::vector<i64> job_start, job_completion;  // -1 = never completed
+  std::vector<Run> runs;                       // order: window, phase, rank
+  std::vector<i64> tau, k;                     // phase table (GBA/GSA) or the single (tau, k)
+  std::vector<i64> n_part;                     // participants per phase, summed over windows
+  i64 flow = 0, horizon = 0, job_steps = 0, n_unfinished = 0;
+};
+
+// One call of Procedure StaggeredPipelineSchedule on `part` (already ordered), shifted by `base`:
+// job with rank r starts at base + floor(r*tau/k) and holds its slot for tau rounds; it completes
+// after o rounds if o <= tau and is killed at the end of the slot otherwise.  SimS differs only
+// in the start rule: batches of k start together every tau rounds.
+// Returns the slot end of the last job (the time the next call may begin).
+i64 run_slice(Schedule& S, const std::vector<i64>& part, const int32_t* s, const int32_t* o,
+              i64 base, i64 tau, i64 k, i64 phase, bool simultaneous) {
+  i64 N = static_cast<i64>(part.size());
+  if (N == 0) return base;
+  for (i64 r = 0; r < N; ++r) {
+    i64 i = part[r];
+    i64 st = simultaneous ? base + (r / k) * tau : base + (r * tau) / k;
+    i64 d = std::min<i64>(o[i], tau);
+    S.runs.push_back(Run{i, phase, st, d, s[i]});
+    if (o[i] <= tau) { S.job_start[i] = st; S.job_completion[i] = st + o[i]; }
+  }
+  i64 last = simultaneous ? ((N - 1) / k) * tau : ((N - 1) * tau) / k;
+  return base + last + tau;
+}
+
+Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int32_t* o_est,
+                const i64* arrival, i64 M, int a, int b, i64 beta0, i64 s_bar_in, i64 tau_in,
+                i64 k_in, i64 window) {
+  Schedule* S = new Schedule();
+  S->n = n;
+  S->job_start.assign(n, -1);
+  S->job_completion.assign(n, -1);
+  if (family < 0 || family > 3 || n < 0 || M < 1 || window < 0 || tau_in < 0 || k_in < 0) {
+    S->status = 3; return S;
+  }
+  i64 s_bar = s_bar_in;
+  if (s_bar < 0) { s_bar = 0; for (i64 i = 0; i < n; ++i) s_bar = std::max<i64>(s_bar, s[i]); }
+  S->s_bar = s_bar;
+  i64 X = M - s_bar;                      // largest response length that fits (per-job feasibility)
+  if (X < 1) { S->status = 1; return S; }
+  for (i64 i = 0; i < n; ++i) {
+    if (o[i] < 1 || s[i] < 0) { S->status = 3; return S; }
+    if (o[i] > X) { S->status = 1; return S; }
+  }
+  if (arrival)
+    for (i64 i = 0; i < n; ++i)
+      if (arrival[i] < 0 || (i > 0 && arrival[i] < arrival[i - 1])) { S->status = 3; return S; }
+  if (window == 0 && arrival)
+    for (i64 i = 0; i < n; ++i) if (arrival[i] != 0) { S->status = 3; return S; }
+
+  const bool geometric = (family == FAM_GBA || family == FAM_GSA);
+  if (geometric) {
+    if (a <= b || b < 1) { S->status = 3; return S; }
+    S->tau = ladder(X, a, b, beta0);
+    for (i64 t : S->tau) S->k.push_back(kstar(t, s_bar, M));
+    S->n_part.assign(S->tau.size(), 0);
+  }
+
+  // Windows: consecutive jobs with the same floor(arrival / window) form one offline sub-instance.
+  std::vector<std::pair<i64, i64>> groups;     // [lo, hi)
+  std::vector<i64> group_release;              // earliest time the group's schedule may begin
+  if (window > 0 && arrival) {
+    i64 lo = 0;
+    while (lo < n) {
+      i64 w = arrival[lo] / window, hi = lo;
+      while (hi < n && arrival[hi] / window == w) ++hi;
+      groups.push_back({lo, hi});
+      group_release.push_back((w + 1) * window);
+      lo = hi;
+    }
+  } else if (n > 0) {
+    groups.push_back({0, n});
+    group_release.push_back(0);
+  }
+
+  i64 base = 0;
+  for (size_t g = 0; g < groups.size(); ++g) {
+    base = std::max(base, group_release[g]);
+    const i64 lo = groups[g].first, hi = groups[g].second;
+    std::vector<i64> order(hi - lo);
+    std::iota(order.begin(), order.end(), lo);
+    const bool keyed = !(family == FAM_GSA && !o_est);   // plain GSA keeps the index order
+    auto key = [&](i64 i) -> i64 { return o_est ? o_est[i] : o[i]; };
+    if (keyed)
+      std::stable_sort(order.begin(), order.end(), [&](i64 x, i64 y) { return key(x) < key(y); });
+
+    if (geometric) {
+      // entered[i]: job has been admitted to some phase; done[i]: job has completed.
+      std::vector<char> entered(hi - lo, family == FAM_GSA ? 1 : 0), done(hi - lo, 0);
+      i64 left = hi - lo;
+      for (size_t p = 0; p < S->tau.size() && left > 0; ++p) {
+        const i64 tau = S->tau[p], k = S->k[p];
+        std::vector<i64> part;
+        for (i64 i : order) {
+          if (!entered[i - lo] && std::min<i64>(std::max<i64>(key(i), 1), X) <= tau) entered[i - lo] = 1;
+          if (entered[i - lo] && !done[i - lo]) part.push_back(i);
+        }
+        S->n_part[p] += static_cast<i64>(part.size());
+        if (k < 1) { S->status = 1; return S; }
+        base = run_slice(*S, part, s, o, base, tau, k, static_cast<i64>(p), false);
+        for (i64 i : part) if (o[i] <= tau) { done[i - lo] = 1; --left; }
+      }
+    } else {
+      i64 tau = tau_in, k = k_in;
+      if (tau == 0) { for (i64 i : order) tau = std::max(tau, key(i)); }
+      if (k == 0) k = (family == FAM_SPS) ? kstar(tau, s_bar, M) : M / (s_bar + tau);
+      if (tau < 1 || k < 1) { S->status = 1; return S; }
+      if (g == 0) { S->tau.push_back(tau); S->k.push_back(k); S->n_part.push_back(0); }
+      S->n_part[0] += hi - lo;
+      base = run_slice(*S, order, s, o, base, tau, k, 0, family == FAM_SIMS);
+    }
+  }
+
+  for (const Run& r : S->runs) {
+    S->horizon = std::max(S->horizon, r.start + r.len);
+    S->job_steps += r.len;
+  }
+  for (i64 i = 0; i < n; ++i) {
+    if (S->job_completion[i] < 0) ++S->n_unfinished;
+    else S->flow += S->job_completion[i] - (arrival ? arrival[i] : 0);
+  }
+  return S;
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---- closed forms -----------------------------------------------------------
+int64_t kvo_peak_closed(int64_t k, int64_t tau, int64_t s) { return peak_closed(k, tau, s); }
+int64_t kvo_kstar(int64_t tau, int64_t s, int64_t M) { return kstar(tau, s, M); }
+
+// Writes up to cap slice lengths; returns the number of phases (may exceed cap), 0 on bad input.
+int64_t kvo_ladder(int64_t X, int32_t a, int32_t b, int64_t beta0, int64_t* tau, int64_t cap) {
+  std::vector<i64> t = ladder(X, a, b, beta0);
+  for (size_t i = 0; i < t.size() && static_cast<i64>(i) < cap; ++i) tau[i] = t[i];
+  return static_cast<i64>(t.size());
+}
+
+// ---- schedule builder -------------------------------------------------------
+void* kvo_build(int32_t family, int64_t n, const int32_t* s, const int32_t* o, const int32_t* o_est,
+                const int64_t* arrival, int64_t M, int32_t alpha_num, int32_t alpha_den,
+                int64_t beta0, int64_t s_bar, int64_t tau, int64_t k, int64_t window) {
+  return build(family, n, s, o, o_est, arrival, M, alpha_num, alpha_den, beta0, s_bar, tau, k, window);
+}
+void kvo_free(void* h) { delete static_cast<Schedule*>(h); }
+
+// scalars: [status, n_runs, n_phases, horizon, flow, job_steps, n_unfinished, s_bar]
+void kvo_scalars(const void* h, int64_t* out) {
+  const Schedule* S = static_cast<const Schedule*>(h);
+  out[0] = S->status; out[1] = static_cast<i64>(S->runs.size()); out[2] = static_cast<i64>(S->tau.size());
+  out[3] = S->horizon; out[4] = S->flow; out[5] = S->job_steps; out[6] = S->n_unfinished; out[7] = S->s_bar;
+}
+void kvo_jobs(const void* h, int64_t* start, int64_t* completion) {
+  const Schedule* S = static_cast<const Schedule*>(h);
+  std::copy(S->job_start.begin(), S->job_start.end(), start);
+  std::copy(S->job_completion.begin(), S->job_completion.end(), completion);
+}
+void kvo_runs(const void* h, int64_t* job, int64_t* phase, int64_t* start, int64_t* len, int64_t* s) {
+  const Schedule* S = static_cast<const Schedule*>(h);
+  for (size_t r = 0; r < S->runs.size(); ++r) {
+    job[r] = S->runs[r].job; phase[r] = S->runs[r].phase; start[r] = S->runs[r].start;
+    len[r] = S->runs[r].len; s[r] = S->runs[r].s;
+  }
+}
+void kvo_phases(const void* h, int64_t* tau, int64_t* k, int64_t* n_part) {
+  const Schedule* S = static_cast<const Schedule*>(h);
+  std::copy(S->tau.begin(), S->tau.end(), tau);
+  std::copy(S->k.begin(), S->k.end(), k);
+  std::copy(S->n_part.begin(), S->n_part.end(), n_part);
+}
+
+// ---- evaluators -------------------------------------------------------------
+// Dense definition: a run (start, len, s) holds s + u + 1 tokens in round start + u, u < len
+// (Eq. Memory-Feasibility).  profile may be NULL; when given it has room for `cap` rounds and
+// rounds beyond cap are not written.  out = [peak, horizon, job_steps, first round of the peak].
+void kvo_eval_dense(int64_t R, const int64_t* start, const int64_t* len, const int64_t* s,
+                    int64_t* profile, int64_t cap, int64_t* out) {
+  i64 T = 0, steps = 0;
+  for (i64 r = 0; r < R; ++r) { T = std::max(T, start[r] + len[r]); steps += len[r]; }
+  std::vector<i64> mem(static_cast<size_t>(T), 0);
+  for (i64 r = 0; r < R; ++r)
+    for (i64 u = 0; u < len[r]; ++u) mem[start[r] + u] += s[r] + u + 1;
+  i64 peak = 0, arg = -1;
+  for (i64 t = 0; t < T; ++t) if (mem[t] > peak) { peak = mem[t]; arg = t; }
+  if (profile) for (i64 t = 0; t < T && t < cap; ++t) profile[t] = mem[t];
+  out[0] = peak; out[1] = T; out[2] = steps; out[3] = arg;
+}
+
+// Event form for horizons too long for a dense array: between two consecutive event times the
+// active set is fixed and each active job grows by one token per round, so the maximum of a
+// segment is at its last round.  out as above (without the arg).
+void kvo_eval_events(int64_t R, const int64_t* start, const int64_t* len, const int64_t* s, int64_t* out) {
+  struct Ev { i64 t, dcount, dconst; };
+  std::vector<Ev> ev;
+  ev.reserve(static_cast<size_t>(2 * R));
+  i64 T = 0, steps = 0;
+  for (i64 r = 0; r < R; ++r) {
+    if (len[r] <= 0) continue;
+    i64 c = s[r] + 1 - start[r];           // tokens at round t are c + t while active
+    ev.push_back(Ev{start[r], +1, +c});
+    ev.push_back(Ev{start[r] + len[r], -1, -c});
+    T = std::max(T, start[r] + len[r]); steps += len[r];
+  }
+  std::sort(ev.begin(), ev.end(), [](const Ev& x, const Ev& y) { return x.t < y.t; });
+  i64 count = 0, cst = 0, peak = 0;
+  for (size_t i = 0; i < ev.size();) {
+    size_t j = i;
+    while (j < ev.size() && ev[j].t == ev[i].t) { count += ev[j].dcount; cst += ev[j].dconst; ++j; }
+    if (j < ev.size() && count > 0) {
+      i64 last = ev[j].t - 1;
+      peak = std::max(peak, cst + count * last);
+    }
+    i = j;
+  }
+  out[0] = peak; out[1] = T; out[2] = steps; out[3] = -1;
+}
+
+// ---- brute-force optimum (tiny instances, identical prompt length) ----------
+// An optimal schedule never kills or pauses, so it is a vector of start rounds; search round by
+// round over which waiting jobs start now.  Jobs with equal response length are started in index
+// order (symmetry).  Returns the minimum total flow time, or -1 if some job cannot fit alone.
+namespace {
+struct Opt {
+  int n; i64 s, M; const int32_t* o; std::vector<i64> mem; i64 best;
+  void dfs(i64 t, unsigned waiting, i64 cost) {
+    if (!waiting) { best = std::min(best, cost); return; }
+    i64 lb = cost;
+    for (int i = 0; i < n; ++i) if (waiting >> i & 1) lb += t + o[i];
+    if (lb >= best) return;
+    bool idle = (static_cast<size_t>(t) >= mem.size()) || mem[t] == 0;
+    for (unsigned sub = waiting;; sub = (sub - 1) & waiting) {
+      bool ok = !(idle && sub == 0);
+      for (int j = 0; ok && j < n; ++j)       // equal lengths start in index order
+        if (sub >> j & 1)
+          for (int i = 0; i < j; ++i)
+            if ((waiting >> i & 1) && !(sub >> i & 1) && o[i] == o[j]) { ok = false; break; }
+      if (ok) {
+        i64 add = 0;
+        for (int i = 0; i < n; ++i) if (sub >> i & 1) {
+          if (mem.size() < static_cast<size_t>(t + o[i])) mem.resize(t + o[i], 0);
+          for (i64 u = 0; u < o[i]; ++u) mem[t + u] += s + u + 1;
+          add += t + o[i];
+        }
+        bool fits = true;
+        for (size_t x = t; x < mem.size(); ++x) if (mem[x] > M) { fits = false; break; }
+        if (fits) dfs(t + 1, waiting & ~sub, cost + add);
+        for (int i = 0; i < n; ++i) if (sub >> i & 1)
+          for (i64 u = 0; u < o[i]; ++u) mem[t + u] -= s + u + 1;
+      }
+      if (sub == 0) break;
+    }
+  }
+};
+}  // namespace
+
+int64_t kvo_opt_bruteforce(int32_t n, int64_t s, const int32_t* o, int64_t M) {
+  if (n < 0 || n > 10) return -1;
+  for (int i = 0; i < n; ++i) if (s + o[i] > M) return -1;
+  Opt opt{n, s, M, o, {}, INT64_MAX};
+  opt.dfs(0, (1u << n) - 1u, 0);
+  return opt.best;
+}
+
+}  // extern "C"
