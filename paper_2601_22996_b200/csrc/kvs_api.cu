@@ -1,0 +1,453 @@
+// C ABI: argument validation, workspace layout, launches.  Host code only.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "kvs_internal.cuh"
+
+struct kvs_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  unsigned char* workspace = nullptr;
+  uint64_t workspace_bytes = 0;
+  int sm_count = 0;
+  int build_ctas_per_sm = 1;
+  bool timing = false;
+  bool timed = false;
+  cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before the ordering kernel, between, after the builder
+  std::string err;
+};
+
+namespace {
+
+constexpr int64_t KVS_MAX_GRID = 1024;        // upper bound on CTAs of the fused kernel (sizes the carry lists)
+constexpr int64_t KVS_TIME_LIMIT = 1ll << 31; // exclusive bound on M, tau, k
+
+int fail(kvs_ctx* ctx, int code, const char* msg) {
+  if (ctx) ctx->err = msg;
+  return code;
+}
+int fail_cuda(kvs_ctx* ctx, cudaError_t e, const char* where) {
+  if (ctx) ctx->err = std::string(where) + ": " + cudaGetErrorString(e);
+  return KVS_E_CUDA;
+}
+
+size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+// Offsets of the scratch regions of the fused path inside the workspace.  Calls are ordered on
+// one stream, so the entry points reuse the workspace from offset 0; the layout without staging
+// is a prefix of the layout with staging.
+struct Layout {
+  size_t settings, stats, perm, perm_tmp, sorted_s, sorted_o, sorted_key, lists;
+  size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
+  size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
+  size_t total;
+};
+
+Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging) {
+  Layout L{};
+  size_t at = 0;
+  auto take = [&](size_t bytes) { size_t r = at; at += align_up(bytes); return r; };
+  L.settings = take(static_cast<size_t>(P) * sizeof(kvs_setting));
+  L.stats = take(static_cast<size_t>(I) * sizeof(InstStats));
+  L.perm = take(static_cast<size_t>(N) * 4);
+  L.perm_tmp = take(static_cast<size_t>(N) * 4);
+  L.sorted_s = take(static_cast<size_t>(N) * 4);
+  L.sorted_o = take(static_cast<size_t>(N) * 4);
+  L.sorted_key = take(static_cast<size_t>(N) * 4);
+  const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
+  L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 4);
+  if (staging) {
+    L.st_off = take(static_cast<size_t>(I + 1) * 8);
+    L.st_s = take(static_cast<size_t>(N) * 4);
+    L.st_o = take(static_cast<size_t>(N) * 4);
+    L.st_key = take(static_cast<size_t>(N) * 4);
+    L.st_arr = take(static_cast<size_t>(N) * 8);
+    L.sc_peak = take(static_cast<size_t>(P) * 8);
+    L.sc_flow = take(static_cast<size_t>(P) * 8);
+    L.sc_steps = take(static_cast<size_t>(P) * 8);
+    L.sc_hor = take(static_cast<size_t>(P) * 8);
+    L.sc_unf = take(static_cast<size_t>(P) * 8);
+    L.sc_feas = take(static_cast<size_t>(P));
+    L.sc_stat = take(static_cast<size_t>(P) * 4);
+  }
+  L.total = at;
+  return L;
+}
+
+// Generic evaluator: 64-bit constant terms and 32-bit slopes, capacity + one slot per evaluation.
+size_t generic_bytes(int64_t cap_total, int64_t P, size_t* second) {
+  const size_t a = align_up(static_cast<size_t>(cap_total + P) * 8);
+  if (second) *second = a;
+  return a + align_up(static_cast<size_t>(cap_total + P) * 4);
+}
+
+struct SweepLayout {
+  size_t stats, perm, perm_tmp, sorted_s, sorted_o, prefix_s, prefix_o, tau, k, acc_peak, acc_flow, total;
+};
+
+SweepLayout make_sweep_layout(int64_t N, int64_t max_n) {
+  SweepLayout L{};
+  size_t at = 0;
+  auto take = [&](size_t bytes) { size_t r = at; at += align_up(bytes); return r; };
+  L.stats = take(sizeof(InstStats));
+  L.perm = take(static_cast<size_t>(N) * 4);
+  L.perm_tmp = take(static_cast<size_t>(N) * 4);
+  L.sorted_s = take(static_cast<size_t>(N) * 4);
+  L.sorted_o = take(static_cast<size_t>(N) * 4);
+  L.prefix_s = take(static_cast<size_t>(max_n + 1) * 8);
+  L.prefix_o = take(static_cast<size_t>(max_n + 1) * 8);
+  L.tau = take(65536 * 8);
+  L.k = take(65536 * 8);
+  L.acc_peak = take(65536 * 8);
+  L.acc_flow = take(65536 * 8);
+  L.total = at;
+  return L;
+}
+
+int check_instances(kvs_ctx* ctx, const kvs_instances* inst) {
+  if (!inst) return fail(ctx, KVS_E_ARG, "instances: null");
+  if (inst->n_instances < 0 || inst->n_jobs_total < 0 || inst->max_jobs_per_instance < 0)
+    return fail(ctx, KVS_E_ARG, "instances: negative size");
+  if (inst->max_jobs_per_instance >= (1ll << 31) - 1) return fail(ctx, KVS_E_RANGE, "instances: more than 2^31-2 jobs in one instance");
+  if (!inst->job_off) return fail(ctx, KVS_E_ARG, "instances: job_off is null");
+  if (inst->n_jobs_total > 0 && (!inst->s || !inst->o)) return fail(ctx, KVS_E_ARG, "instances: s or o is null");
+  if (inst->window < 0) return fail(ctx, KVS_E_ARG, "instances: negative window");
+  if (inst->window == 0 && inst->arrival) return fail(ctx, KVS_E_ARG, "instances: arrival given without a window (offline instances take arrival = NULL)");
+  return KVS_OK;
+}
+
+// The ladder keeps a^j and X*b^j exactly in 128 bits.  With ell = floor(log_alpha X) the largest
+// value formed is below a * X * b^(ell+1) (a^j <= X * b^j up to j = ell, one more factor for the
+// test that ends the search); refuse parameters for which that might not fit, or that need more
+// phases than the table holds.
+bool ladder_fits(int64_t M, int a, int b) {
+  const double la = std::log2(static_cast<double>(a)), lb = std::log2(static_cast<double>(b));
+  const double lx = std::log2(static_cast<double>(M));
+  const double ell = std::floor(lx / (la - lb)) + 1.0;   // one spare for rounding of the logarithms
+  if (ell + 2.0 > KVS_MAX_PHASES) return false;
+  return la + lx + (ell + 2.0) * lb < 125.0;             // also covers beta0 * a^p < a * X * b^p
+}
+
+int check_settings(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* st, int64_t P) {
+  if (P < 0) return fail(ctx, KVS_E_ARG, "settings: negative count");
+  if (P > 0 && !st) return fail(ctx, KVS_E_ARG, "settings: null");
+  for (int64_t e = 0; e < P; ++e) {
+    const kvs_setting& s = st[e];
+    if (s.instance < 0 || s.instance >= inst->n_instances) return fail(ctx, KVS_E_ARG, "settings: instance out of range");
+    if (s.family < KVS_GBA || s.family > KVS_SIMS) return fail(ctx, KVS_E_ARG, "settings: unknown family");
+    if (s.M < 1 || s.M >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: M outside [1, 2^31)");
+    if (s.s_bar < -1) return fail(ctx, KVS_E_ARG, "settings: s_bar < -1");
+    if (s.tau < 0 || s.tau >= KVS_TIME_LIMIT || s.k < 0 || s.k >= KVS_TIME_LIMIT)
+      return fail(ctx, KVS_E_RANGE, "settings: tau or k outside [0, 2^31)");
+    if (s.family == KVS_GBA || s.family == KVS_GSA) {
+      if (s.alpha_den < 1 || s.alpha_num <= s.alpha_den) return fail(ctx, KVS_E_ARG, "settings: alpha must be > 1");
+      if (s.beta0 < 0 || s.beta0 >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: beta0 outside [0, 2^31)");
+      if (!(s.alpha_num == 2 && s.alpha_den == 1) && !ladder_fits(s.M, s.alpha_num, s.alpha_den))
+        return fail(ctx, KVS_E_RANGE, "settings: ladder for this alpha and M needs more than 96 phases or 128-bit integers");
+    }
+  }
+  return KVS_OK;
+}
+
+int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P,
+              const kvs_schedule_out* out, const kvs_eval_out* ev, int do_profile) {
+  if (!ctx) return KVS_E_STATE;
+  int rc = check_instances(ctx, inst);
+  if (rc) return rc;
+  rc = check_settings(ctx, inst, settings, P);
+  if (rc) return rc;
+  kvs_schedule_out o{};
+  kvs_eval_out v{};
+  if (out) o = *out;
+  if (ev) v = *ev;
+  const bool job_out = o.job_start || o.job_completion || o.job_start64 || o.job_completion64;
+  if (job_out && !o.job_out_off) return fail(ctx, KVS_E_ARG, "schedule_out: job outputs need job_out_off");
+  const bool run_out = o.run_job || o.run_phase || o.run_start || o.run_len || o.run_s;
+  if (run_out && !o.run_off) return fail(ctx, KVS_E_ARG, "schedule_out: run outputs need run_off");
+  if (v.profile && !v.profile_off) return fail(ctx, KVS_E_ARG, "eval_out: profile needs profile_off");
+  if (!do_profile) v.profile = nullptr;
+  if (P == 0) return KVS_OK;
+
+  const int64_t N = inst->n_jobs_total, I = inst->n_instances, max_n = inst->max_jobs_per_instance;
+  const Layout L = make_layout(N, I, max_n, P, false);
+  if (L.total > ctx->workspace_bytes)
+    return fail(ctx, KVS_E_CAPACITY, "workspace too small for this call (see kvs_workspace_bytes)");
+  cudaError_t ce = cudaSetDevice(ctx->device);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
+  unsigned char* ws = ctx->workspace;
+  ce = cudaMemcpyAsync(ws + L.settings, settings, static_cast<size_t>(P) * sizeof(kvs_setting), cudaMemcpyHostToDevice, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of settings");
+
+  bool need_order = inst->o_est != nullptr;
+  for (int64_t e = 0; e < P && !need_order; ++e) need_order = settings[e].family != KVS_GSA;
+
+  SortParams sp{};
+  sp.job_off = inst->job_off; sp.s = inst->s; sp.o = inst->o; sp.key = inst->o_est; sp.arrival = inst->arrival;
+  sp.window = inst->window; sp.n_instances = I; sp.max_jobs = max_n; sp.need_order = need_order ? 1 : 0;
+  sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
+  sp.perm = reinterpret_cast<int32_t*>(ws + L.perm);
+  sp.perm_tmp = reinterpret_cast<int32_t*>(ws + L.perm_tmp);
+  sp.sorted_s = reinterpret_cast<int32_t*>(ws + L.sorted_s);
+  sp.sorted_o = reinterpret_cast<int32_t*>(ws + L.sorted_o);
+  sp.sorted_key = reinterpret_cast<int32_t*>(ws + L.sorted_key);
+  const int64_t sort_cap = static_cast<int64_t>(ctx->sm_count) * 2;
+  const int sort_grid = static_cast<int>(I < sort_cap ? I : sort_cap);
+  if (ctx->timing) cudaEventRecord(ctx->ev[0], ctx->stream);
+  ce = kvs_launch_sort(sp, sort_grid, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "sort launch");
+  if (ctx->timing) cudaEventRecord(ctx->ev[1], ctx->stream);
+
+  BuildParams bp{};
+  bp.job_off = inst->job_off; bp.s = inst->s; bp.o = inst->o; bp.key = inst->o_est; bp.arrival = inst->arrival;
+  bp.window = inst->window; bp.n_instances = I; bp.max_jobs = max_n;
+  bp.perm = sp.perm; bp.sorted_s = sp.sorted_s; bp.sorted_o = sp.sorted_o; bp.sorted_key = sp.sorted_key;
+  bp.stats = sp.stats;
+  bp.settings = reinterpret_cast<const kvs_setting*>(ws + L.settings);
+  bp.P = P; bp.out = o; bp.ev = v; bp.do_profile = do_profile;
+  bp.lists = reinterpret_cast<int32_t*>(ws + L.lists);
+  int64_t grid = static_cast<int64_t>(ctx->sm_count) * ctx->build_ctas_per_sm;
+  if (grid > KVS_MAX_GRID) grid = KVS_MAX_GRID;
+  if (grid > P) grid = P;
+  ce = kvs_launch_build(bp, static_cast<int>(grid), ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "build launch");
+  if (ctx->timing) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; }
+  return KVS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int kvs_init(const kvs_init_params* params, kvs_ctx** out) {
+  if (!params || !out) return KVS_E_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0) return KVS_E_CUDA;  // no CPU fallback exists
+  if (params->device < 0 || params->device >= count) return KVS_E_ARG;
+  if (params->workspace_bytes > 0 && !params->workspace) return KVS_E_ARG;
+  if (reinterpret_cast<uintptr_t>(params->workspace) & 255u) return KVS_E_ARG;
+  kvs_ctx* ctx = new (std::nothrow) kvs_ctx();
+  if (!ctx) return KVS_E_STATE;
+  ctx->device = params->device;
+  ctx->stream = static_cast<cudaStream_t>(params->stream);
+  ctx->workspace = static_cast<unsigned char*>(params->workspace);
+  ctx->workspace_bytes = params->workspace_bytes;
+  cudaDeviceProp prop;
+  if (cudaSetDevice(ctx->device) != cudaSuccess || cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) {
+    delete ctx;
+    return KVS_E_CUDA;
+  }
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->build_ctas_per_sm = kvs_build_ctas_per_sm();
+  *out = ctx;
+  return KVS_OK;
+}
+
+int kvs_destroy(kvs_ctx* ctx) {
+  if (ctx)
+    for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
+  delete ctx;
+  return KVS_OK;
+}
+
+const char* kvs_last_error(const kvs_ctx* ctx) { return ctx ? ctx->err.c_str() : "no context"; }
+
+int kvs_set_timing(kvs_ctx* ctx, int32_t enabled) {
+  if (!ctx) return KVS_E_STATE;
+  if (enabled && !ctx->ev[0]) {
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return fail(ctx, KVS_E_CUDA, "cudaSetDevice");
+    for (cudaEvent_t& e : ctx->ev)
+      if (cudaEventCreate(&e) != cudaSuccess) return fail(ctx, KVS_E_CUDA, "cudaEventCreate");
+  }
+  ctx->timing = enabled != 0;
+  ctx->timed = false;
+  return KVS_OK;
+}
+
+int kvs_last_timing(kvs_ctx* ctx, float* sort_ms, float* build_ms) {
+  if (!ctx) return KVS_E_STATE;
+  if (sort_ms) *sort_ms = 0.f;
+  if (build_ms) *build_ms = 0.f;
+  if (!ctx->timed) return KVS_OK;
+  cudaError_t ce = cudaEventSynchronize(ctx->ev[2]);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaEventSynchronize");
+  if (sort_ms) cudaEventElapsedTime(sort_ms, ctx->ev[0], ctx->ev[1]);
+  if (build_ms) cudaEventElapsedTime(build_ms, ctx->ev[1], ctx->ev[2]);
+  return KVS_OK;
+}
+
+int kvs_workspace_bytes(int64_t n_jobs_total, int64_t n_instances, int64_t max_jobs_per_instance,
+                        int64_t n_evaluations, int64_t generic_capacity, int32_t host_staging, uint64_t* out) {
+  if (!out || n_jobs_total < 0 || n_instances < 0 || max_jobs_per_instance < 0 || n_evaluations < 0 || generic_capacity < 0)
+    return KVS_E_ARG;
+  size_t need = make_layout(n_jobs_total, n_instances, max_jobs_per_instance, n_evaluations, host_staging != 0).total;
+  if (generic_capacity > 0) {
+    const size_t g = generic_bytes(generic_capacity, n_evaluations, nullptr);
+    if (g > need) need = g;
+  }
+  const size_t w = make_sweep_layout(n_jobs_total, max_jobs_per_instance).total;
+  if (w > need) need = w;
+  *out = need;
+  return KVS_OK;
+}
+
+int kvs_build_schedule(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P,
+                       const kvs_schedule_out* out, const kvs_eval_out* ev) {
+  return run_fused(ctx, inst, settings, P, out, ev, 0);
+}
+
+int kvs_evaluate_built(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P,
+                       const kvs_schedule_out* out, const kvs_eval_out* ev) {
+  return run_fused(ctx, inst, settings, P, out, ev, 1);
+}
+
+int kvs_evaluate_built_host(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P,
+                            const kvs_eval_out* ev) {
+  if (!ctx) return KVS_E_STATE;
+  int rc = check_instances(ctx, inst);
+  if (rc) return rc;
+  if (!ev) return fail(ctx, KVS_E_ARG, "eval_out: null");
+  if (ev->profile) return fail(ctx, KVS_E_ARG, "host entry point returns scalars only (profile must be NULL)");
+  if (P < 0) return fail(ctx, KVS_E_ARG, "settings: negative count");
+  const int64_t N = inst->n_jobs_total, I = inst->n_instances;
+  const Layout L = make_layout(N, I, inst->max_jobs_per_instance, P, true);
+  if (L.total > ctx->workspace_bytes) return fail(ctx, KVS_E_CAPACITY, "workspace too small for host staging (see kvs_workspace_bytes)");
+  cudaError_t ce = cudaSetDevice(ctx->device);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
+  unsigned char* ws = ctx->workspace;
+  auto h2d = [&](size_t off, const void* src, size_t bytes) {
+    return (src && bytes) ? cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, ctx->stream) : cudaSuccess;
+  };
+  if ((ce = h2d(L.st_off, inst->job_off, static_cast<size_t>(I + 1) * 8)) != cudaSuccess ||
+      (ce = h2d(L.st_s, inst->s, static_cast<size_t>(N) * 4)) != cudaSuccess ||
+      (ce = h2d(L.st_o, inst->o, static_cast<size_t>(N) * 4)) != cudaSuccess ||
+      (ce = h2d(L.st_key, inst->o_est, static_cast<size_t>(N) * 4)) != cudaSuccess ||
+      (ce = h2d(L.st_arr, inst->arrival, static_cast<size_t>(N) * 8)) != cudaSuccess)
+    return fail_cuda(ctx, ce, "host-to-device copy of the instances");
+  kvs_instances dev = *inst;
+  dev.job_off = reinterpret_cast<const int64_t*>(ws + L.st_off);
+  dev.s = reinterpret_cast<const int32_t*>(ws + L.st_s);
+  dev.o = reinterpret_cast<const int32_t*>(ws + L.st_o);
+  dev.o_est = inst->o_est ? reinterpret_cast<const int32_t*>(ws + L.st_key) : nullptr;
+  dev.arrival = inst->arrival ? reinterpret_cast<const int64_t*>(ws + L.st_arr) : nullptr;
+  kvs_eval_out d{};
+  d.peak = reinterpret_cast<int64_t*>(ws + L.sc_peak);
+  d.flow = reinterpret_cast<int64_t*>(ws + L.sc_flow);
+  d.job_steps = reinterpret_cast<int64_t*>(ws + L.sc_steps);
+  d.horizon = reinterpret_cast<int64_t*>(ws + L.sc_hor);
+  d.n_unfinished = reinterpret_cast<int64_t*>(ws + L.sc_unf);
+  d.feasible = reinterpret_cast<uint8_t*>(ws + L.sc_feas);
+  d.status = reinterpret_cast<int32_t*>(ws + L.sc_stat);
+  rc = run_fused(ctx, &dev, settings, P, nullptr, &d, 1);
+  if (rc) return rc;
+  auto d2h = [&](void* dst, size_t off, size_t bytes) {
+    return (dst && bytes) ? cudaMemcpyAsync(dst, ws + off, bytes, cudaMemcpyDeviceToHost, ctx->stream) : cudaSuccess;
+  };
+  const size_t p8 = static_cast<size_t>(P) * 8;
+  if ((ce = d2h(ev->peak, L.sc_peak, p8)) != cudaSuccess || (ce = d2h(ev->flow, L.sc_flow, p8)) != cudaSuccess ||
+      (ce = d2h(ev->job_steps, L.sc_steps, p8)) != cudaSuccess || (ce = d2h(ev->horizon, L.sc_hor, p8)) != cudaSuccess ||
+      (ce = d2h(ev->n_unfinished, L.sc_unf, p8)) != cudaSuccess ||
+      (ce = d2h(ev->feasible, L.sc_feas, static_cast<size_t>(P))) != cudaSuccess ||
+      (ce = d2h(ev->status, L.sc_stat, static_cast<size_t>(P) * 4)) != cudaSuccess)
+    return fail_cuda(ctx, ce, "device-to-host copy of the results");
+  ce = cudaStreamSynchronize(ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "stream synchronize");
+  return KVS_OK;
+}
+
+int kvs_evaluate_schedule(kvs_ctx* ctx, const kvs_runs* runs, const kvs_eval_out* ev) {
+  if (!ctx) return KVS_E_STATE;
+  if (!runs || !ev) return fail(ctx, KVS_E_ARG, "runs or eval_out is null");
+  if (runs->P < 0) return fail(ctx, KVS_E_ARG, "runs: negative count");
+  if (runs->P == 0) return KVS_OK;
+  if (!runs->run_off || !runs->run_start || !runs->run_len || !runs->run_s) return fail(ctx, KVS_E_ARG, "runs: null array");
+  if (!ev->profile_off) return fail(ctx, KVS_E_ARG, "eval_out: profile_off (capacities) is required");
+  cudaError_t ce = cudaSetDevice(ctx->device);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
+  // total capacity = profile_off[P]: one small synchronous read sizes the scratch arrays
+  int64_t cap_total = 0;
+  ce = cudaMemcpyAsync(&cap_total, ev->profile_off + runs->P, 8, cudaMemcpyDeviceToHost, ctx->stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "read of profile_off");
+  if (cap_total < 0) return fail(ctx, KVS_E_ARG, "eval_out: negative capacity");
+  size_t need_a = 0;
+  const size_t need = generic_bytes(cap_total, runs->P, &need_a);
+  if (need > ctx->workspace_bytes) return fail(ctx, KVS_E_CAPACITY, "workspace too small for the generic evaluator");
+  unsigned char* ws = ctx->workspace;
+  GenericParams gp{};
+  gp.runs = *runs; gp.ev = *ev;
+  gp.dconst = reinterpret_cast<i64*>(ws);
+  gp.dcount = reinterpret_cast<int32_t*>(ws + need_a);
+  ce = cudaMemsetAsync(ws, 0, need, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "memset");
+  ce = kvs_launch_generic(gp, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "generic launch");
+  return KVS_OK;
+}
+
+int kvs_sweep(kvs_ctx* ctx, const kvs_instances* inst, const kvs_sweep_params* params, const kvs_sweep_out* out) {
+  if (!ctx) return KVS_E_STATE;
+  int rc = check_instances(ctx, inst);
+  if (rc) return rc;
+  if (!params || !out) return fail(ctx, KVS_E_ARG, "sweep: params or out is null");
+  if (inst->o_est || inst->window != 0) return fail(ctx, KVS_E_ARG, "sweep: needs offline instances ordered by the exact response length");
+  if (params->instance < 0 || params->instance >= inst->n_instances) return fail(ctx, KVS_E_ARG, "sweep: instance out of range");
+  if (params->family != KVS_SPS && params->family != KVS_SIMS) return fail(ctx, KVS_E_ARG, "sweep: family must be SPS or SIMS");
+  if (params->n_tau < 0 || params->n_k < 0 || static_cast<int64_t>(params->n_tau) * params->n_k > 65536)
+    return fail(ctx, KVS_E_RANGE, "sweep: grid larger than 65536 settings");
+  if (params->n_tau == 0 || params->n_k == 0) return KVS_OK;
+  if (!params->tau || !params->k) return fail(ctx, KVS_E_ARG, "sweep: null grid");
+  if (params->M < 1 || params->M >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "sweep: M outside [1, 2^31)");
+  for (int i = 0; i < params->n_tau; ++i)
+    if (params->tau[i] < 1 || params->tau[i] >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "sweep: tau outside [1, 2^31)");
+  for (int i = 0; i < params->n_k; ++i)
+    if (params->k[i] < 1 || params->k[i] >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "sweep: k outside [1, 2^31)");
+  const int64_t N = inst->n_jobs_total, max_n = inst->max_jobs_per_instance;
+  const SweepLayout L = make_sweep_layout(N, max_n);
+  if (L.total > ctx->workspace_bytes) return fail(ctx, KVS_E_CAPACITY, "workspace too small for the sweep (see kvs_workspace_bytes)");
+  cudaError_t ce = cudaSetDevice(ctx->device);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
+  unsigned char* ws = ctx->workspace;
+
+  // order and statistics of the one instance: the sort kernel sees a batch of one
+  SortParams sp{};
+  sp.job_off = inst->job_off + params->instance; sp.s = inst->s; sp.o = inst->o; sp.key = nullptr; sp.arrival = nullptr;
+  sp.window = 0; sp.n_instances = 1; sp.max_jobs = max_n; sp.need_order = 1;
+  sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
+  sp.perm = reinterpret_cast<int32_t*>(ws + L.perm);
+  sp.perm_tmp = reinterpret_cast<int32_t*>(ws + L.perm_tmp);
+  sp.sorted_s = reinterpret_cast<int32_t*>(ws + L.sorted_s);
+  sp.sorted_o = reinterpret_cast<int32_t*>(ws + L.sorted_o);
+  sp.sorted_key = nullptr;
+  ce = kvs_launch_sort(sp, 1, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "sort launch");
+  // the instance's first job index and size are device values; read them once (16 bytes)
+  int64_t range[2] = {0, 0};
+  ce = cudaMemcpyAsync(range, inst->job_off + params->instance, 16, cudaMemcpyDeviceToHost, ctx->stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "read of job_off");
+  const int64_t lo = range[0], n = range[1] - range[0];
+  if (lo < 0 || n < 0 || n > max_n || lo + n > N) return fail(ctx, KVS_E_ARG, "sweep: job_off inconsistent with the stated sizes");
+
+  i64* ps = reinterpret_cast<i64*>(ws + L.prefix_s);
+  i64* po = reinterpret_cast<i64*>(ws + L.prefix_o);
+  ce = kvs_launch_prefix(sp.sorted_s + lo, sp.sorted_o + lo, n, ps, po, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "prefix launch");
+  ce = cudaMemcpyAsync(ws + L.tau, params->tau, static_cast<size_t>(params->n_tau) * 8, cudaMemcpyHostToDevice, ctx->stream);
+  if (ce == cudaSuccess)
+    ce = cudaMemcpyAsync(ws + L.k, params->k, static_cast<size_t>(params->n_k) * 8, cudaMemcpyHostToDevice, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of the grids");
+  SweepParams wp{};
+  wp.sorted_s = sp.sorted_s + lo; wp.sorted_o = sp.sorted_o + lo; wp.prefix_s = ps; wp.prefix_o = po;
+  wp.n = n; wp.family = params->family; wp.M = params->M;
+  wp.tau = reinterpret_cast<const i64*>(ws + L.tau); wp.k = reinterpret_cast<const i64*>(ws + L.k);
+  wp.n_tau = params->n_tau; wp.n_k = params->n_k; wp.out = *out;
+  ce = kvs_launch_sweep(wp, reinterpret_cast<i64*>(ws + L.acc_peak), reinterpret_cast<u64*>(ws + L.acc_flow), ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "sweep launch");
+  return KVS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,163 @@
+// Internal declarations shared by the kernels and the C ABI (not part of the public interface).
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "kvs.h"
+
+typedef int64_t i64;
+typedef uint64_t u64;
+typedef unsigned long long ull;   // the type CUDA's 64-bit atomics are declared on
+typedef unsigned int u32;
+
+constexpr int KVS_MAX_PHASES = 96;      // slices of one geometric ladder
+constexpr int KVS_SORT_THREADS = 1024;  // one CTA sorts one (instance, window) segment at a time
+constexpr int KVS_EVAL_THREADS = 512;   // one CTA per evaluation
+constexpr int KVS_EVAL_ITEMS = 8;       // rounds per thread and tile
+constexpr int KVS_TILE = KVS_EVAL_THREADS * KVS_EVAL_ITEMS;  // rounds per shared-memory tile
+
+// Per-instance statistics produced by the first kernel.
+struct InstStats {
+  int32_t s_max;
+  int32_t o_max;
+  int32_t key_max;
+  int32_t flags;  // KVS_EVAL_BAD_INPUT or 0
+};
+
+// Device view of one call of the fused builder/evaluator.
+struct BuildParams {
+  // instances
+  const i64* job_off;
+  const int32_t* s;
+  const int32_t* o;
+  const int32_t* key;       // estimates, or NULL when the exact o orders and classifies
+  const i64* arrival;
+  i64 window;
+  i64 n_instances;
+  i64 max_jobs;
+  // order by key (per instance and window), produced by the sort kernel
+  const int32_t* perm;      // position -> job index inside the instance
+  const int32_t* sorted_s;
+  const int32_t* sorted_o;
+  const int32_t* sorted_key;
+  const InstStats* stats;
+  // evaluations
+  const kvs_setting* settings;
+  i64 P;
+  kvs_schedule_out out;
+  kvs_eval_out ev;
+  int do_profile;
+  // per-CTA carry lists: 2 * max_jobs entries each
+  int32_t* lists;
+};
+
+struct SortParams {
+  const i64* job_off;
+  const int32_t* s;
+  const int32_t* o;
+  const int32_t* key;       // NULL: sort by o
+  const i64* arrival;
+  i64 window;
+  i64 n_instances;
+  i64 max_jobs;
+  int need_order;           // 0: statistics only
+  InstStats* stats;
+  int32_t* perm;
+  int32_t* perm_tmp;
+  int32_t* sorted_s;
+  int32_t* sorted_o;
+  int32_t* sorted_key;      // written only when key != NULL
+};
+
+struct GenericParams {
+  kvs_runs runs;
+  kvs_eval_out ev;
+  i64* dconst;              // [capacity_total + P] difference array of the constant terms
+  int32_t* dcount;          // [capacity_total + P] difference array of the slopes
+};
+
+struct SweepParams {
+  const int32_t* sorted_s;  // the instance in key order
+  const int32_t* sorted_o;
+  const i64* prefix_s;      // [n + 1]
+  const i64* prefix_o;      // [n + 1]
+  i64 n;
+  int family;
+  i64 M;
+  const i64* tau;           // DEVICE copies of the grids
+  const i64* k;
+  int n_tau, n_k;
+  kvs_sweep_out out;
+};
+
+cudaError_t kvs_launch_sort(const SortParams& p, int grid, cudaStream_t stream);
+cudaError_t kvs_launch_build(const BuildParams& p, int grid, cudaStream_t stream);
+int kvs_build_ctas_per_sm();
+cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
+cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,
+                              i64* prefix_o, cudaStream_t stream);
+cudaError_t kvs_launch_sweep(const SweepParams& p, i64* acc_peak, u64* acc_flow, cudaStream_t stream);
+
+// ---- small device helpers ---------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ u32 lane_id() { return threadIdx.x & 31u; }
+__device__ __forceinline__ u32 lanemask_lt() {
+  u32 m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// floor(r * tau / k) for 0 <= r, tau < 2^31 and 1 <= k < 2^31.
+__device__ __forceinline__ i64 slot_offset(i64 r, i64 tau, i64 k) {
+  u64 x = static_cast<u64>(r) * static_cast<u64>(tau);
+  if ((x >> 32) == 0) return static_cast<i64>(static_cast<u32>(x) / static_cast<u32>(k));
+  return static_cast<i64>(x / static_cast<u64>(k));
+}
+
+__device__ __forceinline__ i64 ceil_div_u(u64 x, u64 y) { return static_cast<i64>((x + y - 1) / y); }
+__device__ __forceinline__ i64 min_i64(i64 x, i64 y) { return x < y ? x : y; }
+__device__ __forceinline__ i64 max_i64(i64 x, i64 y) { return x > y ? x : y; }
+
+template <typename T>
+__device__ __forceinline__ T warp_sum(T v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+  return v;
+}
+template <typename T>
+__device__ __forceinline__ T warp_max(T v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    T w = __shfl_xor_sync(0xffffffffu, v, d);
+    v = w > v ? w : v;
+  }
+  return v;
+}
+
+// Block-wide reductions; `scratch` has room for 32 values; result valid in every thread.
+template <typename T>
+__device__ __forceinline__ T block_sum(T v, T* scratch) {
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane_id() == 0) scratch[threadIdx.x >> 5] = v;
+  __syncthreads();
+  T r = 0;
+  int nw = (blockDim.x + 31) >> 5;
+  if (static_cast<int>(lane_id()) < nw) r = scratch[lane_id()];
+  return warp_sum(r);
+}
+template <typename T>
+__device__ __forceinline__ T block_max(T v, T* scratch, T lowest) {
+  v = warp_max(v);
+  __syncthreads();
+  if (lane_id() == 0) scratch[threadIdx.x >> 5] = v;
+  __syncthreads();
+  T r = lowest;
+  int nw = (blockDim.x + 31) >> 5;
+  if (static_cast<int>(lane_id()) < nw) r = scratch[lane_id()];
+  return warp_max(r);
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,160 @@
+// Per-instance statistics and the stable order of jobs by (estimated) response length.
+//
+// One CTA handles one instance at a time.  It first reduces the instance's statistics
+// (largest prompt, response and key; input validation), then, window by window, sorts the
+// job indices by key with a least-significant-digit radix sort (8-bit digits).  Stability
+// (ties keep the original index order) is what makes the order unique, so that the per-job
+// results agree bit for bit with a stable comparison sort.
+//
+// Each pass ranks one tile of 1024 jobs at a time: lanes with equal digits find each other with
+// a warp match, per-warp digit counts go to shared memory, one column scan per digit turns them
+// into offsets behind the running bucket position.  Keys are re-read through the permutation
+// (they stay in L2 for instances of this size), so only 4 bytes per job move per pass.
+#include "kvs_internal.cuh"
+
+namespace {
+
+constexpr int T = KVS_SORT_THREADS;
+constexpr int WARPS = T / 32;
+
+__device__ __forceinline__ int32_t key_at(const SortParams& p, i64 lo, int idx) {
+  return p.key ? p.key[lo + idx] : p.o[lo + idx];
+}
+
+// Sort positions [seg_lo, seg_hi) of the instance starting at global job index lo.
+__device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
+                             u32 (*warp_cnt)[256], u32* bucket, u32 (*hist)[256]) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int n = seg_hi - seg_lo;
+  int32_t* const out = p.perm + lo + seg_lo;
+  if (passes == 0 || n <= 1) {
+    for (int j = tid; j < n; j += T) out[j] = seg_lo + j;
+    __syncthreads();
+    return;
+  }
+  // digit histograms of all passes in one sweep
+  for (int i = tid; i < 4 * 256; i += T) (&hist[0][0])[i] = 0;
+  __syncthreads();
+  for (int j = tid; j < n; j += T) {
+    u32 key = static_cast<u32>(key_at(p, lo, seg_lo + j));
+    for (int d = 0; d < passes; ++d) atomicAdd(&hist[d][(key >> (8 * d)) & 255u], 1u);
+  }
+  __syncthreads();
+  // exclusive scan of each histogram: warp d scans histogram d, 8 digits per lane
+  if (warp < passes) {
+    u32 v[8], sum = 0;
+    for (int i = 0; i < 8; ++i) { v[i] = hist[warp][lane_id() * 8 + i]; sum += v[i]; }
+    u32 incl = sum;
+    for (int d = 1; d < 32; d <<= 1) {
+      u32 y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (static_cast<int>(lane_id()) >= d) incl += y;
+    }
+    u32 run = incl - sum;
+    for (int i = 0; i < 8; ++i) { hist[warp][lane_id() * 8 + i] = run; run += v[i]; }
+  }
+  __syncthreads();
+
+  for (int pass = 0; pass < passes; ++pass) {
+    // the last pass must land in perm: passes alternate between the two buffers
+    const bool to_perm = ((passes - 1 - pass) & 1) == 0;
+    int32_t* dst = (to_perm ? p.perm : p.perm_tmp) + lo + seg_lo;
+    const int32_t* src = (to_perm ? p.perm_tmp : p.perm) + lo + seg_lo;
+    if (tid < 256) bucket[tid] = hist[pass][tid];
+    for (int j0 = 0; j0 < n; j0 += T) {
+      for (int i = tid; i < WARPS * 256; i += T) (&warp_cnt[0][0])[i] = 0;
+      __syncthreads();
+      const int j = j0 + tid;
+      const bool valid = j < n;
+      int idx = 0;
+      u32 digit = 256;  // sentinel for lanes past the end
+      if (valid) {
+        idx = pass == 0 ? seg_lo + j : src[j];
+        digit = (static_cast<u32>(key_at(p, lo, idx)) >> (8 * pass)) & 255u;
+      }
+      const u32 peers = __match_any_sync(0xffffffffu, digit);
+      const u32 rank = __popc(peers & lanemask_lt());
+      if (valid && rank == 0) warp_cnt[warp][digit] = __popc(peers);
+      __syncthreads();
+      if (tid < 256) {
+        u32 acc = bucket[tid];
+        for (int w = 0; w < WARPS; ++w) {
+          u32 t = warp_cnt[w][tid];
+          warp_cnt[w][tid] = acc;
+          acc += t;
+        }
+        bucket[tid] = acc;
+      }
+      __syncthreads();
+      if (valid) dst[warp_cnt[warp][digit] + rank] = idx;
+      __syncthreads();
+    }
+  }
+}
+
+__global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
+  __shared__ u32 warp_cnt[WARPS][256];
+  __shared__ u32 hist[4][256];
+  __shared__ u32 bucket[256];
+  __shared__ int red[32];
+  __shared__ int seg_end;
+  const int tid = threadIdx.x;
+
+  for (i64 inst = blockIdx.x; inst < p.n_instances; inst += gridDim.x) {
+    const i64 lo = p.job_off[inst], hi = p.job_off[inst + 1];
+    int flags = 0;
+    if (hi < lo || hi - lo > p.max_jobs) flags = KVS_EVAL_BAD_INPUT;
+    const int n = flags ? 0 : static_cast<int>(hi - lo);
+    int s_max = 0, o_max = 0, key_max = 0, bad = 0;
+    for (int j = tid; j < n; j += T) {
+      const int sv = p.s[lo + j], ov = p.o[lo + j], kv = key_at(p, lo, j);
+      s_max = max(s_max, sv); o_max = max(o_max, ov); key_max = max(key_max, kv);
+      bad |= (sv < 0) | (ov < 1) | (kv < 1);
+      if (p.arrival) {
+        const i64 a = p.arrival[lo + j];
+        bad |= (a < 0) | (j > 0 && p.arrival[lo + j - 1] > a);
+      }
+    }
+    s_max = block_max(s_max, red, 0);
+    o_max = block_max(o_max, red, 0);
+    key_max = block_max(key_max, red, 0);
+    bad = block_max(bad, red, 0);
+    if (bad) flags = KVS_EVAL_BAD_INPUT;
+    if (tid == 0) p.stats[inst] = InstStats{s_max, o_max, key_max, flags};
+    if (!p.need_order || flags) continue;  // uniform across the CTA
+
+    const int passes = key_max > 0 ? (32 - __clz(key_max) + 7) / 8 : 0;
+    int seg_lo = 0;
+    while (seg_lo < n) {
+      if (tid == 0) {
+        int end = n;
+        if (p.window > 0 && p.arrival) {  // first position whose arrival falls in a later window
+          const i64 limit = (p.arrival[lo + seg_lo] / p.window + 1) * p.window;
+          int a = seg_lo + 1, b = n;
+          while (a < b) { int m = (a + b) >> 1; if (p.arrival[lo + m] < limit) a = m + 1; else b = m; }
+          end = a;
+        }
+        seg_end = end;
+      }
+      __syncthreads();
+      const int seg_hi = seg_end;
+      sort_segment(p, lo, seg_lo, seg_hi, passes, warp_cnt, bucket, hist);
+      __syncthreads();
+      for (int j = seg_lo + tid; j < seg_hi; j += T) {
+        const int idx = p.perm[lo + j];
+        p.sorted_s[lo + j] = p.s[lo + idx];
+        p.sorted_o[lo + j] = p.o[lo + idx];
+        if (p.key) p.sorted_key[lo + j] = p.key[lo + idx];
+      }
+      __syncthreads();
+      seg_lo = seg_hi;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t kvs_launch_sort(const SortParams& p, int grid, cudaStream_t stream) {
+  if (p.n_instances <= 0) return cudaSuccess;
+  k_stats_sort<<<grid, KVS_SORT_THREADS, 0, stream>>>(p);
+  return cudaGetLastError();
+}

@@ -1,0 +1,186 @@
+// Parameter sweep: SPS or the simultaneous schedule for every (tau, k) of a grid on one
+// instance, scalars only.  Horizons reach billions of rounds, so nothing dense is formed.
+//
+// Jobs are in key order (key = exact response length), rank i starts at floor(i*tau/k)
+// (Procedure StaggeredPipelineSchedule) or floor(i/k)*tau (simultaneous batches) and runs
+// d_i = min(o_i, tau) rounds.  Starts and run lengths are both nondecreasing in i, hence so are
+// the run ends, and the jobs active in round t are a contiguous index range [e, b).  Memory is
+// piecewise linear and increasing between events, so its maximum is attained in the last round
+// of some run, t = end_i - 1, where
+//     memory(t) = sum_{j in [i, b)} (s_j + t - start_j + 1)
+//               = PS_s[b] - PS_s[i] + (b - i)(t + 1) - sum_{j in [i, b)} start_j
+// with b = #{j : start_j <= t} = min(n, ceil((t+1)k/tau))  (the count c(rho) in the proof of Lemma
+// "Peak Memory Usage of SPS").  Using i instead of the first index with the same end can only
+// drop non-negative terms, and that first index is itself a candidate, so the maximum is exact.
+// Each thread walks consecutive candidates, sliding the window sum of starts; long jumps of b use
+// the closed form sum_{j<n} floor(j*tau/k) (Euclid-like floor sum).
+#include "kvs_internal.cuh"
+
+namespace {
+
+constexpr int SW_THREADS = 128;
+constexpr int SW_PER = 64;
+constexpr int SW_CHUNK = SW_THREADS * SW_PER;
+
+// sum_{j=0}^{n-1} floor((a*j + b) / m), arithmetic modulo 2^64
+__device__ u64 floor_sum(u64 n, u64 m, u64 a, u64 b) {
+  u64 ans = 0;
+  for (;;) {
+    if (a >= m) { ans += (n - 1) * n / 2 * (a / m); a %= m; }
+    if (b >= m) { ans += n * (b / m); b %= m; }
+    const u64 y = a * n + b;
+    if (y < m) break;
+    n = y / m;
+    b = y % m;
+    const u64 t = m; m = a; a = t;
+  }
+  return ans;
+}
+
+__global__ void __launch_bounds__(SW_THREADS) k_sweep(SweepParams p, i64 n_chunks, i64* acc_peak, u64* acc_flow) {
+  __shared__ i64 red64[32];
+  const i64 setting = blockIdx.x / n_chunks, chunk = blockIdx.x % n_chunks;
+  const i64 tau = p.tau[setting / p.n_k], k = p.k[setting % p.n_k];
+  const i64 n = p.n;
+  const i64 i0 = chunk * SW_CHUNK + static_cast<i64>(threadIdx.x) * SW_PER;
+  const i64 i1 = i0 + SW_PER < n ? i0 + SW_PER : n;
+  i64 peak = 0;
+  u64 flow = 0;
+  if (i0 < n) {
+    if (p.family == KVS_SPS) {
+      const i64 qt = tau / k, rt = tau % k;
+      u64 x = static_cast<u64>(i0) * static_cast<u64>(tau);
+      i64 qi = static_cast<i64>(x / static_cast<u64>(k)), ri = static_cast<i64>(x % static_cast<u64>(k));
+      i64 b = i0, qb = qi, rb = ri;   // b: first job not yet counted as started; (qb, rb): its start and remainder
+      u64 W = 0;                      // sum of starts over [i, b)
+      for (i64 i = i0; i < i1; ++i) {
+        const i64 oi = p.sorted_o[i];
+        const i64 d = oi < tau ? oi : tau;
+        const i64 t = qi + d - 1;     // last round of run i
+        if (oi <= tau) flow += static_cast<u64>(qi + oi);
+        int steps = 0;
+        while (b < n && qb <= t) {
+          if (steps == 32) {          // long jump: closed forms instead of stepping
+            i64 bn = ceil_div_u(static_cast<u64>(t + 1) * static_cast<u64>(k), static_cast<u64>(tau));
+            if (bn > n) bn = n;
+            W += floor_sum(bn, k, tau, 0) - floor_sum(b, k, tau, 0);
+            b = bn;
+            x = static_cast<u64>(b) * static_cast<u64>(tau);
+            qb = static_cast<i64>(x / static_cast<u64>(k)); rb = static_cast<i64>(x % static_cast<u64>(k));
+            break;
+          }
+          W += static_cast<u64>(qb);
+          ++b; rb += rt; qb += qt;
+          if (rb >= k) { rb -= k; ++qb; }
+          ++steps;
+        }
+        const i64 mem = (p.prefix_s[b] - p.prefix_s[i]) + (b - i) * (t + 1) - static_cast<i64>(W);
+        peak = mem > peak ? mem : peak;
+        W -= static_cast<u64>(qi);
+        ri += rt; qi += qt;
+        if (ri >= k) { ri -= k; ++qi; }
+      }
+    } else {
+      i64 j = i0 / k, rem = i0 % k;   // batch index and position inside the batch
+      for (i64 i = i0; i < i1; ++i) {
+        const i64 oi = p.sorted_o[i];
+        const i64 d = oi < tau ? oi : tau;
+        if (oi <= tau) flow += static_cast<u64>(j * tau + oi);
+        i64 bend = (j + 1) * k;
+        if (bend > n) bend = n;
+        const i64 mem = (p.prefix_s[bend] - p.prefix_s[i]) + (bend - i) * d;   // round start + d - 1 of the batch
+        peak = mem > peak ? mem : peak;
+        if (++rem == k) { rem = 0; ++j; }
+      }
+    }
+  }
+  peak = block_max(peak, red64, static_cast<i64>(0));
+  const i64 fsum = block_sum(static_cast<i64>(flow), red64);
+  if (threadIdx.x == 0) {
+    if (peak > 0) atomicMax(reinterpret_cast<long long*>(acc_peak + setting), static_cast<long long>(peak));
+    if (fsum != 0) atomicAdd(reinterpret_cast<ull*>(acc_flow + setting), static_cast<ull>(fsum));
+  }
+}
+
+__global__ void k_sweep_finish(SweepParams p, const i64* acc_peak, const u64* acc_flow) {
+  const i64 setting = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (setting >= static_cast<i64>(p.n_tau) * p.n_k) return;
+  const i64 tau = p.tau[setting / p.n_k], k = p.k[setting % p.n_k];
+  const i64 n = p.n;
+  i64 a = 0, b = n;                 // completed jobs = those with o <= tau: a prefix in key order
+  while (a < b) { const i64 m = (a + b) >> 1; if (p.sorted_o[m] <= tau) a = m + 1; else b = m; }
+  const i64 c = a;
+  i64 horizon = 0;
+  if (n > 0) {
+    const i64 last = n - 1;
+    const i64 start = p.family == KVS_SPS ? slot_offset(last, tau, k) : (last / k) * tau;
+    const i64 ol = p.sorted_o[last];
+    horizon = start + (ol < tau ? ol : tau);
+  }
+  if (p.out.peak) p.out.peak[setting] = acc_peak[setting];
+  if (p.out.flow) p.out.flow[setting] = static_cast<i64>(acc_flow[setting]);
+  if (p.out.n_completed) p.out.n_completed[setting] = c;
+  if (p.out.horizon) p.out.horizon[setting] = horizon;
+  if (p.out.job_steps) p.out.job_steps[setting] = p.prefix_o[c] + (n - c) * tau;
+  if (p.out.feasible) p.out.feasible[setting] = acc_peak[setting] <= p.M ? 1 : 0;
+}
+
+// Exclusive prefix sums of s and o in key order (one CTA, tile after tile).
+__global__ void __launch_bounds__(1024) k_prefix(const int32_t* s, const int32_t* o, i64 n, i64* ps, i64* po) {
+  __shared__ i64 ws[32], wo[32];
+  i64 run_s = 0, run_o = 0;
+  const int tid = threadIdx.x;
+  if (tid == 0) { ps[0] = 0; po[0] = 0; }
+  for (i64 j0 = 0; j0 < n; j0 += 1024) {
+    const i64 j = j0 + tid;
+    const i64 vs = j < n ? s[j] : 0, vo = j < n ? o[j] : 0;
+    i64 is = vs, io = vo;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const i64 ys = __shfl_up_sync(0xffffffffu, is, d), yo = __shfl_up_sync(0xffffffffu, io, d);
+      if (static_cast<int>(lane_id()) >= d) { is += ys; io += yo; }
+    }
+    __syncthreads();
+    if (lane_id() == 31) { ws[tid >> 5] = is; wo[tid >> 5] = io; }
+    __syncthreads();
+    i64 a = ws[lane_id()], b = wo[lane_id()];
+    i64 ia = a, ib = b;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const i64 ya = __shfl_up_sync(0xffffffffu, ia, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
+      if (static_cast<int>(lane_id()) >= d) { ia += ya; ib += yb; }
+    }
+    const i64 off_s = run_s + __shfl_sync(0xffffffffu, ia - a, tid >> 5);
+    const i64 off_o = run_o + __shfl_sync(0xffffffffu, ib - b, tid >> 5);
+    if (j < n) { ps[j + 1] = off_s + is; po[j + 1] = off_o + io; }
+    run_s += __shfl_sync(0xffffffffu, ia, 31);
+    run_o += __shfl_sync(0xffffffffu, ib, 31);
+  }
+}
+
+}  // namespace
+
+cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,
+                              i64* prefix_o, cudaStream_t stream) {
+  k_prefix<<<1, 1024, 0, stream>>>(sorted_s, sorted_o, n, prefix_s, prefix_o);
+  return cudaGetLastError();
+}
+
+cudaError_t kvs_launch_sweep(const SweepParams& p, i64* acc_peak, u64* acc_flow, cudaStream_t stream) {
+  const i64 n_set = static_cast<i64>(p.n_tau) * p.n_k;
+  if (n_set <= 0) return cudaSuccess;
+  cudaError_t e = cudaMemsetAsync(acc_peak, 0, static_cast<size_t>(n_set) * 8, stream);
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(acc_flow, 0, static_cast<size_t>(n_set) * 8, stream);
+  if (e != cudaSuccess) return e;
+  const i64 n_chunks = (p.n + SW_CHUNK - 1) / SW_CHUNK;
+  if (n_chunks > 0) {
+    const i64 blocks = n_set * n_chunks;
+    if (blocks >= (static_cast<i64>(1) << 31)) return cudaErrorInvalidConfiguration;
+    k_sweep<<<static_cast<unsigned>(blocks), SW_THREADS, 0, stream>>>(p, n_chunks, acc_peak, acc_flow);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  k_sweep_finish<<<static_cast<unsigned>((n_set + 255) / 256), 256, 0, stream>>>(p, acc_peak, acc_flow);
+  return cudaGetLastError();
+}
