@@ -193,6 +193,24 @@ typedef struct {
  * profile_off[P] back to the host once (one small synchronous copy). */
 int kvs_evaluate_schedule(kvs_ctx* ctx, const kvs_runs* runs, const kvs_eval_out* ev);
 
+/* (No counterpart in the paper: a packaging variant of kvs_evaluate_schedule.)
+ * For callers that must not allocate device memory at all - code that runs where cudaMalloc is
+ * forbidden or unavailable, such as a plugin inside a serving process whose memory pool owns the
+ * whole GPU, or a latency-critical loop that may not touch the allocator - and therefore cannot
+ * provide a workspace.  The two difference arrays live in a fixed 12 MiB array inside the library
+ * image (every GPU that loads the library holds it until the process exits).  No context is
+ * needed; `device` and `stream` are given directly, `capacity_total` is the host copy of
+ * profile_off[P].  Limit: capacity_total + P <= 1,048,576, otherwise KVS_E_CAPACITY and a message
+ * in `err` (optional buffer of err_len bytes).  The call itself allocates nothing (no cudaMalloc,
+ * no cudaFree, no allocating library routine).
+ * The first call on each device looks up the array's device address; make that first call
+ * before any stream capture.  All calls on a device share the array: each call clears the part
+ * it uses, so results do not depend on earlier calls, but calls that overlap on the GPU (two
+ * streams, two threads) race - serialise them.  Outputs and status bits as kvs_evaluate_schedule. */
+int kvs_evaluate_schedule_noalloc(int32_t device, void* stream, const kvs_runs* runs,
+                                  const kvs_eval_out* ev, int64_t capacity_total,
+                                  char* err, uint64_t err_len);
+
 /* Parameter sweep on one instance: SPS or SIMS for every (tau, k) of a grid, scalars only. */
 typedef struct {
   int64_t instance;

@@ -71,7 +71,8 @@ class _SweepOut(Structure):
 
 
 EXPORTS = ["kvs_init", "kvs_destroy", "kvs_last_error", "kvs_set_timing", "kvs_last_timing", "kvs_workspace_bytes",
-           "kvs_build_schedule", "kvs_evaluate_built", "kvs_evaluate_built_host", "kvs_evaluate_schedule", "kvs_sweep"]
+           "kvs_build_schedule", "kvs_evaluate_built", "kvs_evaluate_built_host", "kvs_evaluate_schedule", "kvs_sweep",
+           "kvs_evaluate_schedule_noalloc"]
 
 _lib = None
 
@@ -97,8 +98,28 @@ def load(path: str | None = None):
         L.kvs_evaluate_built_host.argtypes = [c_void_p, POINTER(_Instances), c_void_p, c_int64, POINTER(_EvalOut)]
         L.kvs_evaluate_schedule.argtypes = [c_void_p, POINTER(_Runs), POINTER(_EvalOut)]
         L.kvs_sweep.argtypes = [c_void_p, POINTER(_Instances), POINTER(_SweepParams), POINTER(_SweepOut)]
+        L.kvs_evaluate_schedule_noalloc.argtypes = [c_int32, c_void_p, POINTER(_Runs), POINTER(_EvalOut), c_int64,
+                                                    ctypes.c_char_p, c_uint64]
         _lib = L
     return _lib
+
+
+def evaluate_schedule_noalloc(runs: dict, ev: dict, capacity_total: int, device: int | None = None):
+    """kvs_evaluate_schedule_noalloc: evaluates explicit runs without a context or a workspace.
+
+    For callers that may not allocate on the GPU: the scratch is a fixed array inside the library
+    (capacity_total + P <= 1,048,576).  Runs on the current CUDA stream; calls on one device must
+    not overlap.  ``runs`` / ``ev`` as in ``Context.evaluate_schedule``."""
+    dev = torch.cuda.current_device() if device is None else device
+    P = int(runs["run_off"].numel()) - 1
+    cr = _Runs(P, _p(runs["run_off"]), _p(runs["run_start"]), _p(runs["run_len"]), _p(runs["run_s"]),
+               _p(runs.get("run_flow")), _p(runs.get("M")))
+    eo = _EvalOut(*[_p(ev.get(f[0])) for f in _EvalOut._fields_])
+    msg = ctypes.create_string_buffer(256)
+    rc = load().kvs_evaluate_schedule_noalloc(dev, c_void_p(torch.cuda.current_stream(dev).cuda_stream),
+                                              ctypes.byref(cr), ctypes.byref(eo), capacity_total, msg, 256)
+    if rc:
+        raise KvsError(rc, msg.value.decode())
 
 
 def make_settings(rows) -> np.ndarray:

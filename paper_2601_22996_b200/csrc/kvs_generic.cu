@@ -6,6 +6,8 @@
 // in global memory (64-bit constant terms, 32-bit slopes), prefix-sums both tile by tile and
 // forms memory(t) = A(t) + t * B(t), its maximum, and the scalar reductions.  Nothing is assumed
 // about the order or overlap of the runs, so this path trades speed for generality.
+#include <cstdio>
+
 #include "kvs_internal.cuh"
 
 namespace {
@@ -131,4 +133,64 @@ cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream) {
   const int grid = static_cast<int>(p.runs.P < 4096 ? p.runs.P : 4096);
   k_generic_eval<<<grid, T, 0, stream>>>(p);
   return cudaGetLastError();
+}
+
+// ---- variant without any caller- or library-allocated scratch -----------------------------------
+//
+// Same kernel, but the two difference arrays live in a fixed array that is part of the loaded
+// library image on every GPU (12 MiB per device, held until the process exits).  The array is
+// shared by all calls on a device and keeps what the previous call left, so each call clears the
+// part it uses first; two calls that overlap on the GPU would race on it.
+
+constexpr int64_t KVS_NOALLOC_SLOTS = int64_t(1) << 20;   // rounds + evaluations per call
+static __device__ __align__(256) unsigned char kvs_noalloc_scratch[KVS_NOALLOC_SLOTS * 12];
+
+namespace {
+constexpr int KVS_NOALLOC_MAX_DEVICES = 64;
+void* g_noalloc_ptr[KVS_NOALLOC_MAX_DEVICES] = {};   // device address of the array, per device
+void put_msg(char* err, uint64_t len, const char* msg) {
+  if (err && len) { snprintf(err, static_cast<size_t>(len), "%s", msg); }
+}
+}  // namespace
+
+extern "C" int kvs_evaluate_schedule_noalloc(int32_t device, void* stream, const kvs_runs* runs,
+                                             const kvs_eval_out* ev, int64_t capacity_total,
+                                             char* err, uint64_t err_len) {
+  if (!runs || !ev) { put_msg(err, err_len, "runs or eval_out is null"); return KVS_E_ARG; }
+  if (runs->P < 0 || capacity_total < 0) { put_msg(err, err_len, "negative size"); return KVS_E_ARG; }
+  if (device < 0 || device >= KVS_NOALLOC_MAX_DEVICES) { put_msg(err, err_len, "device ordinal out of range"); return KVS_E_ARG; }
+  if (runs->P == 0) return KVS_OK;
+  if (!runs->run_off || !runs->run_start || !runs->run_len || !runs->run_s || !ev->profile_off) {
+    put_msg(err, err_len, "null run array or profile_off");
+    return KVS_E_ARG;
+  }
+  if (capacity_total + runs->P > KVS_NOALLOC_SLOTS) {
+    put_msg(err, err_len, "capacity_total + P exceeds the 1,048,576 slots of the built-in scratch array; "
+                          "use kvs_evaluate_schedule with a workspace instead");
+    return KVS_E_CAPACITY;
+  }
+  cudaError_t ce = cudaSetDevice(device);
+  if (ce != cudaSuccess) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
+  if (!g_noalloc_ptr[device]) {
+    // In host code the array's name is only a handle; its device address has to be asked for,
+    // once per device, with that device current.
+    void* ptr = nullptr;
+    ce = cudaGetSymbolAddress(&ptr, kvs_noalloc_scratch);
+    if (ce != cudaSuccess || !ptr) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
+    g_noalloc_ptr[device] = ptr;
+  }
+  unsigned char* base = static_cast<unsigned char*>(g_noalloc_ptr[device]);
+  const size_t slots = static_cast<size_t>(capacity_total + runs->P);
+  const size_t bytes_a = (slots * 8 + 255) & ~static_cast<size_t>(255);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  ce = cudaMemsetAsync(base, 0, bytes_a + slots * 4, s);   // what must start at zero
+  if (ce != cudaSuccess) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
+  GenericParams gp{};
+  gp.runs = *runs;
+  gp.ev = *ev;
+  gp.dconst = reinterpret_cast<i64*>(base);
+  gp.dcount = reinterpret_cast<int32_t*>(base + bytes_a);
+  ce = kvs_launch_generic(gp, s);
+  if (ce != cudaSuccess) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
+  return KVS_OK;
 }
