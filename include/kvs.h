@@ -139,7 +139,7 @@ typedef struct {
 typedef struct {
   const int64_t* profile_off;   /* DEVICE [P + 1]: capacity offsets into `profile`; an evaluation with
                                    capacity 0 gets no profile (its peak is still computed) */
-  int32_t* profile;             /* DEVICE: tokens held in rounds 0 .. horizon-1 (clipped at the capacity);
+  int32_t* profile;             /* DEVICE, 16-byte aligned: tokens held in rounds 0 .. horizon-1 (clipped at the capacity);
                                    rounds between the horizon and the last slot end, if inside the
                                    capacity, are written as 0 */
   int64_t* peak;                /* DEVICE [P]: max over rounds of the profile (-1 if not computed) */

@@ -40,7 +40,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // one stream, so the entry points reuse the workspace from offset 0; the layout without staging
 // is a prefix of the layout with staging.
 struct Layout {
-  size_t settings, stats, perm, perm_tmp, sorted_s, sorted_o, sorted_key, lists;
+  size_t settings, stats, perm, perm_tmp, sorted_s, sorted_o, sorted_key, lists, counter;
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -59,6 +59,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.sorted_key = take(static_cast<size_t>(N) * 4);
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
   L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 4);
+  L.counter = take(8);
   if (staging) {
     L.st_off = take(static_cast<size_t>(I + 1) * 8);
     L.st_s = take(static_cast<size_t>(N) * 4);
@@ -168,6 +169,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   const bool run_out = o.run_job || o.run_phase || o.run_start || o.run_len || o.run_s;
   if (run_out && !o.run_off) return fail(ctx, KVS_E_ARG, "schedule_out: run outputs need run_off");
   if (v.profile && !v.profile_off) return fail(ctx, KVS_E_ARG, "eval_out: profile needs profile_off");
+  if (reinterpret_cast<uintptr_t>(v.profile) & 15u) return fail(ctx, KVS_E_ARG, "eval_out: profile must be 16-byte aligned");
   if (!do_profile) v.profile = nullptr;
   if (P == 0) return KVS_OK;
 
@@ -208,6 +210,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.settings = reinterpret_cast<const kvs_setting*>(ws + L.settings);
   bp.P = P; bp.out = o; bp.ev = v; bp.do_profile = do_profile;
   bp.lists = reinterpret_cast<int32_t*>(ws + L.lists);
+  bp.counter = reinterpret_cast<ull*>(ws + L.counter);
   int64_t grid = static_cast<int64_t>(ctx->sm_count) * ctx->build_ctas_per_sm;
   if (grid > KVS_MAX_GRID) grid = KVS_MAX_GRID;
   if (grid > P) grid = P;

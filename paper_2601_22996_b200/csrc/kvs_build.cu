@@ -10,10 +10,14 @@
 //      compacted list kept in an L2-resident scratch buffer.  Rank r starts at
 //      base + floor(r*tau/k) (Procedure StaggeredPipelineSchedule) or base + floor(r/k)*tau
 //      (simultaneous batches), runs min(o, tau) rounds, completes iff o <= tau;
-//   3. builds the per-round memory of the phase tile by tile in shared memory from two
-//      difference arrays - the constant term s+1-start and the slope 1 of every active run -
-//      each prefix-summed once, memory(t) = A(t) + t*B(t) (Eq. Memory-Feasibility), reduces the
-//      peak, and streams the profile out;
+//   3. walks the rounds of the phase tile by tile.  Ranks start in nondecreasing rounds, so the
+//      runs that start inside a tile are a contiguous rank range and every run is visited exactly
+//      once: its start and completion are written, it is appended to the carry list if killed, and
+//      its two events go into the difference arrays - the constant term s+1-start and the slope 1 -
+//      of the current tile or of the next one (a two-tile ring in shared memory; only slices longer
+//      than a tile need a second look for ends that land further ahead).  Each array is
+//      prefix-summed once, memory(t) = A(t) + t*B(t) (Eq. Memory-Feasibility), the peak is reduced
+//      and the profile is stored straight from registers, 16 bytes at a time;
 //   4. reduces flow time, job-steps, horizon and the number of unfinished jobs.
 //
 // The difference arrays and their sums are kept modulo 2^32.  Every intermediate may wrap, the
@@ -24,9 +28,12 @@
 namespace {
 
 constexpr int T = KVS_EVAL_THREADS;
-constexpr int ITEMS = KVS_EVAL_ITEMS;
+constexpr int ITEMS = KVS_EVAL_ITEMS;      // 8 rounds per thread and tile: two 16-byte vectors
 constexpr int TILE = KVS_TILE;
 constexpr int WARPS = T / 32;
+constexpr int RPT = 4;                     // consecutive ranks per thread in the run loop
+constexpr int CHUNK = T * RPT;
+static_assert(ITEMS == 8, "tile layout assumes two 4-word vectors per thread");
 
 typedef unsigned __int128 u128;
 
@@ -45,9 +52,13 @@ __device__ i64 max_parallelism(i64 tau, i64 s, i64 M) {
   return (k1 * D <= 2 * M - tau + gcd_i64(tau, k1)) ? k1 : k0;
 }
 
+// Shared-memory word of round e of a tile.  Thread t owns rounds 8t .. 8t+7 as two 4-word vectors;
+// vector c of thread t sits at vector index c*T + t, so a warp's vector access is contiguous.
+__device__ __forceinline__ int slot(int e) { return ((((e >> 2) & 1) * T + (e >> 3)) << 2) + (e & 3); }
+
 struct Shared {
-  u32 dA[TILE];             // difference array of constant terms, then the finished profile tile
-  u32 dB[TILE];             // difference array of slopes
+  uint4 dA[2][TILE / 4];    // two-tile ring: difference arrays of the constant terms
+  uint4 dB[2][TILE / 4];    //                and of the slopes
   i64 tau[KVS_MAX_PHASES];
   i64 k[KVS_MAX_PHASES];
   int ent[KVS_MAX_PHASES + 1];  // class boundaries in key order: entrants of phase p are [ent[p], ent[p+1])
@@ -58,7 +69,27 @@ struct Shared {
   int red32[32];
   int n_phases;
   int seg_end;
+  i64 next_eval;
 };
+
+// Adds (c, one) at word idx for every lane with idx >= 0.  With `combine`, lanes of a warp that
+// target the same word (runs that start or end in the same round - thousands of them in a short
+// slice with high parallelism) are summed first, so the word receives one atomic per warp.
+__device__ __forceinline__ void add_event(u32* dA, u32* dB, int idx, u32 c, u32 one, bool combine) {
+  if (combine) {
+    const u32 peers = __match_any_sync(0xffffffffu, idx);
+    if (idx >= 0) {
+      const u32 csum = __reduce_add_sync(peers, c);
+      if ((peers & lanemask_lt()) == 0) {
+        atomicAdd(&dA[idx], csum);
+        atomicAdd(&dB[idx], one * static_cast<u32>(__popc(peers)));
+      }
+    }
+  } else if (idx >= 0) {
+    atomicAdd(&dA[idx], c);
+    atomicAdd(&dB[idx], one);
+  }
+}
 
 // Geometric ladder by warp 0.  Leaves the number of phases in sh.n_phases (0 = too many).
 __device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_bar, i64 M) {
@@ -105,23 +136,27 @@ __device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_b
   __syncwarp();
 }
 
-// Exclusive block scan of a 0/1 flag; returns this thread's offset, total in *total.
-__device__ __forceinline__ int block_flag_scan(bool flag, int* red32, int* total) {
-  const u32 ballot = __ballot_sync(0xffffffffu, flag);
-  const int warp = threadIdx.x >> 5;
-  __syncthreads();
-  if (lane_id() == 0) red32[warp] = __popc(ballot);
-  __syncthreads();
-  int v = (lane_id() < WARPS) ? red32[lane_id()] : 0;
+// Exclusive block scan of a small per-thread count; returns this thread's offset, total in *total.
+__device__ __forceinline__ int block_count_scan(int v, int* red32, int* total) {
   int incl = v;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
-    int y = __shfl_up_sync(0xffffffffu, incl, d);
+    const int y = __shfl_up_sync(0xffffffffu, incl, d);
     if (static_cast<int>(lane_id()) >= d) incl += y;
   }
-  const int warp_off = __shfl_sync(0xffffffffu, incl - v, warp);
-  *total = __shfl_sync(0xffffffffu, incl, 31);
-  return warp_off + __popc(ballot & lanemask_lt());
+  const int warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane_id() == 31) red32[warp] = incl;
+  __syncthreads();
+  const int w = (lane_id() < WARPS) ? red32[lane_id()] : 0;
+  int wi = w;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, wi, d);
+    if (static_cast<int>(lane_id()) >= d) wi += y;
+  }
+  *total = __shfl_sync(0xffffffffu, wi, 31);
+  return __shfl_sync(0xffffffffu, wi - w, warp) + (incl - v);
 }
 
 struct Acc {
@@ -130,14 +165,228 @@ struct Acc {
   u32 peak = 0;
 };
 
-__global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) {
+// Everything one phase needs that does not change while it runs.
+struct Phase {
+  i64 base, tau, k, t_end;
+  int N, C, ent_lo, ph, seg_lo;
+  bool simultaneous, geometric, may_carry, profile_on, combine;
+};
+
+// Per-evaluation pointers and output windows.
+struct EvalCtx {
+  const int32_t* S;       // prompt lengths in schedule order (of the instance)
+  const int32_t* O;       // response lengths in schedule order
+  const int32_t* PERM;    // schedule order -> job index inside the instance, or NULL (identity)
+  const i64* ARR;         // arrivals of the instance, or NULL
+  i64 job_out;            // offset of the evaluation's per-job block
+  i64 run_base, run_cap, run_count;
+  i64 prof_base, prof_cap;
+  bool want_runs;
+};
+
+// Visits ranks [ra, rb) of a phase once: outputs, carry list, and (if the profile is on) the two
+// events of every run.  All of these runs start inside the tile with origin t0; `buf` is the ring
+// half of that tile.  Returns the new length of the carry list.
+__device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
+                                            const int32_t* cur, int32_t* nxt, int C_next, i64 ra, i64 rb,
+                                            i64 t0, int buf, Acc& acc) {
+  const int tid = threadIdx.x;
+  u32* const dA = reinterpret_cast<u32*>(sh.dA);
+  u32* const dB = reinterpret_cast<u32*>(sh.dB);
+  const i64 qt = P.tau / P.k, rt = P.tau % P.k;
+  for (i64 c0 = ra; c0 < rb; c0 += CHUNK) {
+    const i64 r_first = c0 + static_cast<i64>(tid) * RPT;
+    i64 q = 0, rem = 0;   // start offset of the current rank and the remainder that advances it
+    if (r_first < rb) {
+      if (P.simultaneous) { q = (r_first / P.k) * P.tau; rem = r_first % P.k; }
+      else {
+        const u64 x = static_cast<u64>(r_first) * static_cast<u64>(P.tau);
+        if ((x >> 32) == 0) { q = static_cast<u32>(x) / static_cast<u32>(P.k); rem = static_cast<u32>(x) % static_cast<u32>(P.k); }
+        else { q = static_cast<i64>(x / static_cast<u64>(P.k)); rem = static_cast<i64>(x % static_cast<u64>(P.k)); }
+      }
+    }
+    int cpos[RPT];
+    u32 cmask = 0;
+#pragma unroll
+    for (int j = 0; j < RPT; ++j) {
+      const i64 r = r_first + j;
+      int sidx = -1, eidx = -1;
+      u32 c = 0;
+      cpos[j] = 0;
+      if (r < rb) {
+        const int pos = r < P.C ? cur[r] : P.ent_lo + static_cast<int>(r - P.C);
+        const int oi = ec.O[P.seg_lo + pos], si = ec.S[P.seg_lo + pos];
+        const i64 start = P.base + q;
+        const i64 d = oi < P.tau ? oi : P.tau;
+        const bool fin = oi <= P.tau;
+        acc.steps += d;
+        acc.hmax = max_i64(acc.hmax, start + d);
+        if (fin || !P.geometric || ec.want_runs) {
+          const int orig = ec.PERM ? ec.PERM[P.seg_lo + pos] : P.seg_lo + pos;
+          if (fin) {
+            const i64 done = start + oi;
+            acc.flow += done - (ec.ARR ? ec.ARR[orig] : 0);
+            if (p.out.job_start) p.out.job_start[ec.job_out + orig] = static_cast<int32_t>(start);
+            if (p.out.job_completion) p.out.job_completion[ec.job_out + orig] = static_cast<int32_t>(done);
+            if (p.out.job_start64) p.out.job_start64[ec.job_out + orig] = start;
+            if (p.out.job_completion64) p.out.job_completion64[ec.job_out + orig] = done;
+          } else if (!P.geometric) {
+            ++acc.unfinished;
+            if (p.out.job_start) p.out.job_start[ec.job_out + orig] = -1;
+            if (p.out.job_completion) p.out.job_completion[ec.job_out + orig] = -1;
+            if (p.out.job_start64) p.out.job_start64[ec.job_out + orig] = -1;
+            if (p.out.job_completion64) p.out.job_completion64[ec.job_out + orig] = -1;
+          }
+          if (ec.want_runs && ec.run_count + r < ec.run_cap) {
+            const i64 w = ec.run_base + ec.run_count + r;
+            if (p.out.run_job) p.out.run_job[w] = orig;
+            if (p.out.run_phase) p.out.run_phase[w] = P.ph;
+            if (p.out.run_start) p.out.run_start[w] = start;
+            if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
+            if (p.out.run_s) p.out.run_s[w] = si;
+          }
+        }
+        if (!fin && P.geometric) { cpos[j] = pos; cmask |= 1u << j; }
+        if (P.profile_on) {
+          c = static_cast<u32>(si + 1) - static_cast<u32>(start);   // tokens(t) = c + t while active
+          const int srel = static_cast<int>(start - t0);
+          sidx = buf * TILE + slot(srel);
+          if (start + d < P.t_end) {                                  // an end at the phase end is never read
+            const i64 erel = srel + d;
+            if (erel < TILE) eidx = buf * TILE + slot(static_cast<int>(erel));
+            else if (erel < 2 * TILE) eidx = (buf ^ 1) * TILE + slot(static_cast<int>(erel - TILE));
+          }
+        }
+        if (P.simultaneous) { if (++rem == P.k) { rem = 0; q += P.tau; } }
+        else { rem += rt; q += qt; if (rem >= P.k) { rem -= P.k; ++q; } }
+      }
+      if (P.profile_on) {
+        add_event(dA, dB, sidx, c, 1u, P.combine);
+        add_event(dA, dB, eidx, 0u - c, 0xffffffffu, P.combine);
+      }
+    }
+    if (P.may_carry) {
+      int total;
+      int off = C_next + block_count_scan(__popc(cmask), sh.red32, &total);
+#pragma unroll
+      for (int j = 0; j < RPT; ++j)
+        if (cmask >> j & 1u) nxt[off++] = cpos[j];
+      C_next += total;
+    }
+  }
+  return C_next;
+}
+
+// Prefix-sums one tile of the ring, turns it into memory(t), reduces the peak, stores the profile
+// and leaves the tile zeroed for its next use.  Contains one __syncthreads.
+__device__ __forceinline__ void scan_tile(Shared& sh, int buf, i64 t0, int wlen, i64 first_round,
+                                          u32& A_run, u32& B_run, Acc& acc, const EvalCtx& ec, int32_t* profile) {
+  const int tid = threadIdx.x;
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  const uint4 a0 = sh.dA[buf][tid], a1 = sh.dA[buf][T + tid];
+  const uint4 b0 = sh.dB[buf][tid], b1 = sh.dB[buf][T + tid];
+  sh.dA[buf][tid] = zero; sh.dA[buf][T + tid] = zero;
+  sh.dB[buf][tid] = zero; sh.dB[buf][T + tid] = zero;
+  u32 a[ITEMS] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+  u32 b[ITEMS] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+  for (int i = 1; i < ITEMS; ++i) { a[i] += a[i - 1]; b[i] += b[i - 1]; }
+  const u32 sa = a[ITEMS - 1], sb = b[ITEMS - 1];
+  u32 ia = sa, ib = sb;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 ya = __shfl_up_sync(0xffffffffu, ia, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
+    if (static_cast<int>(lane_id()) >= d) { ia += ya; ib += yb; }
+  }
+  if (lane_id() == 31) { sh.redA[tid >> 5] = ia; sh.redB[tid >> 5] = ib; }
+  __syncthreads();
+  const u32 wa = (lane_id() < WARPS) ? sh.redA[lane_id()] : 0, wb = (lane_id() < WARPS) ? sh.redB[lane_id()] : 0;
+  u32 wia = wa, wib = wb;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 ya = __shfl_up_sync(0xffffffffu, wia, d), yb = __shfl_up_sync(0xffffffffu, wib, d);
+    if (static_cast<int>(lane_id()) >= d) { wia += ya; wib += yb; }
+  }
+  const u32 offA = A_run + __shfl_sync(0xffffffffu, wia - wa, tid >> 5) + (ia - sa);
+  const u32 offB = B_run + __shfl_sync(0xffffffffu, wib - wb, tid >> 5) + (ib - sb);
+  A_run += __shfl_sync(0xffffffffu, wia, 31);
+  B_run += __shfl_sync(0xffffffffu, wib, 31);
+  const int e0 = tid * ITEMS;
+  const u32 tt = static_cast<u32>(t0) + static_cast<u32>(e0);
+  u32 mem[ITEMS];
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    mem[i] = (offA + a[i]) + (tt + i) * (offB + b[i]);
+    if (e0 + i < wlen) acc.peak = max(acc.peak, mem[i]);
+  }
+  if (ec.prof_cap > 0) {
+    // rounds [lo, hi) of this tile belong to the phase and fit the caller's capacity
+    const i64 lo = first_round, hi = min_i64(t0 + wlen, ec.prof_cap);
+#pragma unroll
+    for (int v = 0; v < 2; ++v) {
+      const i64 rs = t0 + e0 + 4 * v;
+      int32_t* dst = profile + ec.prof_base + rs;
+      if (rs >= lo && rs + 4 <= hi) {
+        *reinterpret_cast<int4*>(dst) = make_int4(static_cast<int>(mem[4 * v]), static_cast<int>(mem[4 * v + 1]),
+                                                  static_cast<int>(mem[4 * v + 2]), static_cast<int>(mem[4 * v + 3]));
+      } else if (rs + 4 > lo && rs < hi) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (rs + i >= lo && rs + i < hi) dst[i] = static_cast<int>(mem[4 * v + i]);
+      }
+    }
+  }
+}
+
+// Slices longer than a tile: ends that land two or more tiles after the run's start were not
+// inserted when the run was visited; pick them up when their tile comes.
+__device__ __forceinline__ void insert_far_ends(Shared& sh, const EvalCtx& ec, const Phase& P, const int32_t* cur,
+                                                i64 t0_first, i64 t0, int wlen, int buf) {
+  const i64 u0 = t0 - P.base;
+  if (u0 <= TILE) return;
+  const i64 lo = u0 > P.tau ? u0 - P.tau : 0, hi = u0 - TILE;   // start offsets of the candidates: [lo, hi)
+  i64 r_lo, r_hi;
+  if (P.simultaneous) { r_lo = ceil_div_u(lo, P.tau) * P.k; r_hi = ceil_div_u(hi, P.tau) * P.k; }
+  else { r_lo = ceil_div_u(static_cast<u64>(lo) * P.k, P.tau); r_hi = ceil_div_u(static_cast<u64>(hi) * P.k, P.tau); }
+  if (r_hi > P.N) r_hi = P.N;
+  u32* const dA = reinterpret_cast<u32*>(sh.dA);
+  u32* const dB = reinterpret_cast<u32*>(sh.dB);
+  for (i64 r0 = r_lo; r0 < r_hi; r0 += T) {
+    const i64 r = r0 + threadIdx.x;
+    int eidx = -1;
+    u32 c = 0;
+    if (r < r_hi) {
+      const int pos = r < P.C ? cur[r] : P.ent_lo + static_cast<int>(r - P.C);
+      const int oi = ec.O[P.seg_lo + pos], si = ec.S[P.seg_lo + pos];
+      const i64 start = P.base + (P.simultaneous ? (r / P.k) * P.tau : slot_offset(r, P.tau, P.k));
+      const i64 end = start + (oi < P.tau ? oi : P.tau);
+      const i64 ts = t0_first + ((start - t0_first) / TILE) * TILE;   // origin of the tile the run started in
+      if (end >= ts + 2 * TILE && end >= t0 && end < t0 + wlen && end < P.t_end) {
+        c = static_cast<u32>(si + 1) - static_cast<u32>(start);
+        eidx = buf * TILE + slot(static_cast<int>(end - t0));
+      }
+    }
+    add_event(dA, dB, eidx, 0u - c, 0xffffffffu, false);
+  }
+}
+
+__global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   const int tid = threadIdx.x;
   int32_t* const list0 = p.lists + static_cast<i64>(blockIdx.x) * 2 * p.max_jobs;
   int32_t* const list1 = list0 + p.max_jobs;
+  {  // the ring starts zeroed and every tile leaves its half zeroed
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 2 * (TILE / 4); i += T) { (&sh.dA[0][0])[i] = zero; (&sh.dB[0][0])[i] = zero; }
+  }
 
-  for (i64 e = blockIdx.x; e < p.P; e += gridDim.x) {
+  for (;;) {
+    __syncthreads();  // previous evaluation done with shared memory
+    if (tid == 0) sh.next_eval = static_cast<i64>(atomicAdd(reinterpret_cast<ull*>(p.counter), 1ull));
+    __syncthreads();
+    const i64 e = sh.next_eval;
+    if (e >= p.P) break;
     const kvs_setting st = p.settings[e];
     const i64 lo = p.job_off[st.instance];
     const InstStats stats = p.stats[st.instance];
@@ -149,34 +398,34 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) 
     const bool geometric = family == KVS_GBA || family == KVS_GSA;
     const bool simultaneous = family == KVS_SIMS;
     const bool keyed = !(family == KVS_GSA && p.key == nullptr);  // plain GSA keeps the index order
-    const bool may_carry = geometric && (family == KVS_GSA || p.key != nullptr);
-    const int32_t* const S = (keyed ? p.sorted_s : p.s) + lo;
-    const int32_t* const O = (keyed ? p.sorted_o : p.o) + lo;
-    const int32_t* const PERM = keyed ? p.perm + lo : nullptr;
-    const int32_t* const KEY = p.key ? p.sorted_key + lo : O;
+    const int32_t* const KEY = p.key ? p.sorted_key + lo : p.sorted_o + lo;
+
+    EvalCtx ec;
+    ec.S = (keyed ? p.sorted_s : p.s) + lo;
+    ec.O = (keyed ? p.sorted_o : p.o) + lo;
+    ec.PERM = keyed ? p.perm + lo : nullptr;
+    ec.ARR = p.arrival ? p.arrival + lo : nullptr;
+    ec.job_out = p.out.job_out_off ? p.out.job_out_off[e] : 0;
+    ec.run_base = p.out.run_off ? p.out.run_off[e] : 0;
+    ec.run_cap = p.out.run_off ? p.out.run_off[e + 1] - ec.run_base : 0;
+    ec.want_runs = p.out.run_off && (p.out.run_job || p.out.run_phase || p.out.run_start || p.out.run_len || p.out.run_s);
+    ec.prof_base = p.ev.profile_off ? p.ev.profile_off[e] : 0;
+    ec.prof_cap = (p.ev.profile && p.ev.profile_off) ? p.ev.profile_off[e + 1] - ec.prof_base : 0;
+    ec.run_count = 0;
+    const bool want32 = p.out.job_start || p.out.job_completion;
 
     int status = stats.flags;
     if (!status && (X < 1 || stats.o_max > X)) status = KVS_EVAL_INFEASIBLE;
-    __syncthreads();  // previous evaluation done with shared memory
     if (!status && geometric) {
       if (tid < 32) build_ladder(sh, X, st.alpha_num, st.alpha_den, st.beta0, s_bar, M);
       __syncthreads();
       if (sh.n_phases == 0) status = KVS_EVAL_RANGE;
     }
-
-    const i64 job_out = p.out.job_out_off ? p.out.job_out_off[e] : 0;
-    const bool want32 = p.out.job_start || p.out.job_completion;
-    const i64 run_base = p.out.run_off ? p.out.run_off[e] : 0;
-    const i64 run_cap = p.out.run_off ? p.out.run_off[e + 1] - run_base : 0;
-    const bool want_runs = p.out.run_off && (p.out.run_job || p.out.run_phase || p.out.run_start || p.out.run_len || p.out.run_s);
-    const i64 prof_base = p.ev.profile_off ? p.ev.profile_off[e] : 0;
-    const i64 prof_cap = (p.ev.profile && p.ev.profile_off) ? p.ev.profile_off[e + 1] - prof_base : 0;
     bool profile_on = p.do_profile != 0;
 
     Acc acc;
     i64 base = 0;          // first round of the next phase
     i64 written_to = 0;    // profile rounds [0, written_to) have been written
-    i64 run_count = 0;
 
     int seg_lo = 0;
     while (!status && seg_lo < n) {
@@ -184,9 +433,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) 
       if (tid == 0) {
         int end = n;
         if (p.window > 0 && p.arrival) {
-          const i64 limit = (p.arrival[lo + seg_lo] / p.window + 1) * p.window;
+          const i64 limit = (ec.ARR[seg_lo] / p.window + 1) * p.window;
           int a = seg_lo + 1, b = n;
-          while (a < b) { int m = (a + b) >> 1; if (p.arrival[lo + m] < limit) a = m + 1; else b = m; }
+          while (a < b) { int m = (a + b) >> 1; if (ec.ARR[m] < limit) a = m + 1; else b = m; }
           end = a;
         }
         sh.seg_end = end;
@@ -194,15 +443,12 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) 
       __syncthreads();
       const int seg_hi = sh.seg_end;
       const int nseg = seg_hi - seg_lo;
-      if (p.window > 0 && p.arrival) {
-        const i64 release = (p.arrival[lo + seg_lo] / p.window + 1) * p.window;
-        base = max_i64(base, release);
-      }
+      if (p.window > 0 && p.arrival) base = max_i64(base, (ec.ARR[seg_lo] / p.window + 1) * p.window);
 
       int L = 1;
       if (geometric) {
         L = sh.n_phases;
-        // class boundaries: entrants of phase p have clip(key) <= tau_p and > tau_(p-1)
+        // class boundaries: entrants of phase q-1 have clip(key) <= tau_(q-1) and > tau_(q-2)
         for (int q = tid; q <= L; q += T) {
           int v;
           if (q == 0) v = 0;
@@ -232,144 +478,48 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) 
         const int ent_lo = sh.ent[ph], ent_hi = sh.ent[ph + 1];
         const int N = C + (ent_hi - ent_lo);
         if (N == 0) continue;          // an empty class takes no time
-        const i64 tau = sh.tau[ph], k = sh.k[ph];
-        const i64 len = (simultaneous ? ((N - 1) / k) * tau : slot_offset(N - 1, tau, k)) + tau;
+        Phase P;
+        P.base = base; P.tau = sh.tau[ph]; P.k = sh.k[ph];
+        P.N = N; P.C = C; P.ent_lo = ent_lo; P.ph = ph; P.seg_lo = seg_lo;
+        P.simultaneous = simultaneous; P.geometric = geometric;
+        P.may_carry = geometric && (family == KVS_GSA || p.key != nullptr);
+        P.combine = simultaneous ? P.k >= 4 : P.k >= 2 * P.tau;  // several runs per round: combine equal targets within a warp
+        const i64 len = (simultaneous ? ((N - 1) / P.k) * P.tau : slot_offset(N - 1, P.tau, P.k)) + P.tau;
+        P.t_end = base + len;
+        if (profile_on && min_i64(N, P.k + 1) * (static_cast<i64>(stats.s_max) + P.tau) >= (static_cast<i64>(1) << 32)) {
+          profile_on = false;
+          status |= KVS_EVAL_RANGE;
+        }
+        P.profile_on = profile_on;
 
-        // ---- pass A: starts, completions, carry list ----
         int C_next = 0;
-        for (int r0 = 0; r0 < N; r0 += T) {
-          const int r = r0 + tid;
-          bool carry = false;
-          int pos = 0;
-          if (r < N) {
-            pos = r < C ? cur[r] : ent_lo + (r - C);
-            const int oi = O[seg_lo + pos], si = S[seg_lo + pos];
-            const i64 start = base + (simultaneous ? (r / k) * tau : slot_offset(r, tau, k));
-            const i64 d = oi < tau ? oi : tau;
-            const bool fin = oi <= tau;
-            acc.steps += d;
-            acc.hmax = max_i64(acc.hmax, start + d);
-            const int orig = PERM ? PERM[seg_lo + pos] : seg_lo + pos;
-            if (fin) {
-              const i64 done = start + oi;
-              acc.flow += done - (p.arrival ? p.arrival[lo + orig] : 0);
-              if (p.out.job_start) p.out.job_start[job_out + orig] = static_cast<int32_t>(start);
-              if (p.out.job_completion) p.out.job_completion[job_out + orig] = static_cast<int32_t>(done);
-              if (p.out.job_start64) p.out.job_start64[job_out + orig] = start;
-              if (p.out.job_completion64) p.out.job_completion64[job_out + orig] = done;
-            } else if (!geometric) {
-              ++acc.unfinished;
-              if (p.out.job_start) p.out.job_start[job_out + orig] = -1;
-              if (p.out.job_completion) p.out.job_completion[job_out + orig] = -1;
-              if (p.out.job_start64) p.out.job_start64[job_out + orig] = -1;
-              if (p.out.job_completion64) p.out.job_completion64[job_out + orig] = -1;
-            } else {
-              carry = true;
-            }
-            if (want_runs && run_count + r < run_cap) {
-              const i64 w = run_base + run_count + r;
-              if (p.out.run_job) p.out.run_job[w] = orig;
-              if (p.out.run_phase) p.out.run_phase[w] = ph;
-              if (p.out.run_start) p.out.run_start[w] = start;
-              if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
-              if (p.out.run_s) p.out.run_s[w] = si;
-            }
-          }
-          if (may_carry) {
-            int total;
-            const int off = block_flag_scan(carry, sh.red32, &total);
-            if (carry) nxt[C_next + off] = pos;
-            C_next += total;
-          }
-        }
-        run_count += N;
-
-        // ---- pass B: per-round memory of rounds [base, base + len) ----
-        if (profile_on) {
-          const i64 active = min_i64(N, k + 1);
-          if (active * (static_cast<i64>(stats.s_max) + tau) >= (static_cast<i64>(1) << 32)) {
-            profile_on = false;
-            status |= KVS_EVAL_RANGE;
-          }
-        }
-        if (profile_on) {
+        if (!profile_on) {
+          C_next = process_runs(p, sh, ec, P, cur, nxt, 0, 0, N, 0, 0, acc);
+        } else {
           // idle rounds before this phase (window release) hold nothing
-          if (prof_cap > 0)
-            for (i64 t = written_to + tid; t < base && t < prof_cap; t += T) p.ev.profile[prof_base + t] = 0;
+          if (ec.prof_cap > 0)
+            for (i64 t = written_to + tid; t < base && t < ec.prof_cap; t += T) p.ev.profile[ec.prof_base + t] = 0;
+          // tile origins keep the profile stores 16-byte aligned
+          const i64 t0_first = base - ((ec.prof_base + base) & 3);
           u32 A_run = 0, B_run = 0;
-          const i64 t_end = base + len;
-          for (i64 t0 = base; t0 < t_end; t0 += TILE) {
+          i64 r_next = 0;
+          int buf = 0;
+          for (i64 t0 = t0_first; t0 < P.t_end; t0 += TILE) {
+            const int wlen = static_cast<int>(min_i64(TILE, P.t_end - t0));
+            const i64 u_hi = t0 + wlen - base;   // ranks starting before this offset belong to tiles up to this one
+            i64 r_b = simultaneous ? ceil_div_u(u_hi, P.tau) * P.k
+                                   : ceil_div_u(static_cast<u64>(u_hi) * static_cast<u64>(P.k), P.tau);
+            if (r_b > N) r_b = N;
+            C_next = process_runs(p, sh, ec, P, cur, nxt, C_next, r_next, r_b, t0, buf, acc);
+            r_next = r_b;
+            if (P.tau > TILE) insert_far_ends(sh, ec, P, cur, t0_first, t0, wlen, buf);
             __syncthreads();
-#pragma unroll
-            for (int i = 0; i < ITEMS; ++i) { sh.dA[tid + i * T] = 0; sh.dB[tid + i * T] = 0; }
-            __syncthreads();
-            const i64 u0 = t0 - base;
-            const int wlen = static_cast<int>(min_i64(TILE, t_end - t0));
-            const i64 v0 = u0 > tau ? u0 - tau : 0;   // runs ending in this tile started at or after v0
-            i64 r_lo, r_hi;
-            if (simultaneous) {
-              r_lo = ceil_div_u(v0, tau) * k;
-              r_hi = ceil_div_u(u0 + wlen, tau) * k;
-            } else {
-              r_lo = ceil_div_u(static_cast<u64>(v0) * k, tau);
-              r_hi = ceil_div_u(static_cast<u64>(u0 + wlen) * k, tau);
-            }
-            if (r_hi > N) r_hi = N;
-            for (i64 r = r_lo + tid; r < r_hi; r += T) {
-              const int pos = r < C ? cur[r] : ent_lo + static_cast<int>(r - C);
-              const int oi = O[seg_lo + pos], si = S[seg_lo + pos];
-              const i64 start = base + (simultaneous ? (r / k) * tau : slot_offset(r, tau, k));
-              const i64 d = oi < tau ? oi : tau;
-              const u32 c = static_cast<u32>(si + 1) - static_cast<u32>(start);  // tokens(t) = c + t while active
-              const i64 srel = start - t0, erel = srel + d;
-              if (srel >= 0) { atomicAdd(&sh.dA[srel], c); atomicAdd(&sh.dB[srel], 1u); }
-              if (erel >= 0 && erel < wlen) { atomicAdd(&sh.dA[erel], 0u - c); atomicAdd(&sh.dB[erel], 0xffffffffu); }
-            }
-            __syncthreads();
-            // prefix sums of both arrays: thread owns ITEMS consecutive rounds
-            u32 a[ITEMS], b[ITEMS];
-            u32 sa = 0, sb = 0;
-#pragma unroll
-            for (int i = 0; i < ITEMS; ++i) {
-              sa += sh.dA[tid * ITEMS + i]; sb += sh.dB[tid * ITEMS + i];
-              a[i] = sa; b[i] = sb;
-            }
-            u32 ia = sa, ib = sb;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-              const u32 ya = __shfl_up_sync(0xffffffffu, ia, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
-              if (static_cast<int>(lane_id()) >= d) { ia += ya; ib += yb; }
-            }
-            if (lane_id() == 31) { sh.redA[tid >> 5] = ia; sh.redB[tid >> 5] = ib; }
-            __syncthreads();
-            u32 wa = (lane_id() < WARPS) ? sh.redA[lane_id()] : 0, wb = (lane_id() < WARPS) ? sh.redB[lane_id()] : 0;
-            u32 wia = wa, wib = wb;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-              const u32 ya = __shfl_up_sync(0xffffffffu, wia, d), yb = __shfl_up_sync(0xffffffffu, wib, d);
-              if (static_cast<int>(lane_id()) >= d) { wia += ya; wib += yb; }
-            }
-            const u32 offA = A_run + __shfl_sync(0xffffffffu, wia - wa, tid >> 5) + (ia - sa);
-            const u32 offB = B_run + __shfl_sync(0xffffffffu, wib - wb, tid >> 5) + (ib - sb);
-            A_run += __shfl_sync(0xffffffffu, wia, 31);
-            B_run += __shfl_sync(0xffffffffu, wib, 31);
-            const u32 tt = static_cast<u32>(t0) + static_cast<u32>(tid * ITEMS);
-#pragma unroll
-            for (int i = 0; i < ITEMS; ++i) {
-              const u32 mem = (offA + a[i]) + (tt + i) * (offB + b[i]);
-              if (tid * ITEMS + i < wlen) acc.peak = max(acc.peak, mem);
-              sh.dA[tid * ITEMS + i] = mem;
-            }
-            __syncthreads();
-            if (prof_cap > 0)
-              for (int i = tid; i < wlen; i += T) {
-                const i64 t = t0 + i;
-                if (t < prof_cap) p.ev.profile[prof_base + t] = static_cast<int32_t>(sh.dA[i]);
-              }
+            scan_tile(sh, buf, t0, wlen, base, A_run, B_run, acc, ec, p.ev.profile);
+            buf ^= 1;
           }
-          written_to = t_end;
+          written_to = P.t_end;
         }
-
+        ec.run_count += N;
         base += len;
         __syncthreads();               // carry list complete before it is read as `cur`
         int32_t* tmp = cur; cur = nxt; nxt = tmp;
@@ -389,8 +539,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) 
       const bool skipped = (status & (KVS_EVAL_INFEASIBLE | KVS_EVAL_BAD_INPUT)) != 0;
       if (!skipped) {
         if (want32 && hmax > 0x7fffffffll) status |= KVS_EVAL_RANGE;
-        if (want_runs && run_count > run_cap) status |= KVS_EVAL_CAPACITY;
-        if (prof_cap > 0 && hmax > prof_cap) status |= KVS_EVAL_CAPACITY;   // capacity 0 = profile not wanted
+        if (ec.want_runs && ec.run_count > ec.run_cap) status |= KVS_EVAL_CAPACITY;
+        if (ec.prof_cap > 0 && hmax > ec.prof_cap) status |= KVS_EVAL_CAPACITY;   // capacity 0 = profile not wanted
       }
       const bool have_peak = p.do_profile && profile_on && !skipped;
       if (p.ev.peak) p.ev.peak[e] = have_peak ? static_cast<i64>(peak) : -1;
@@ -400,7 +550,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS) k_build_eval(BuildParams p) 
       if (p.ev.n_unfinished) p.ev.n_unfinished[e] = unfinished;
       if (p.ev.feasible) p.ev.feasible[e] = (have_peak && !(status & KVS_EVAL_RANGE) && static_cast<i64>(peak) <= M) ? 1 : 0;
       if (p.ev.status) p.ev.status[e] = status;
-      if (p.out.n_runs) p.out.n_runs[e] = run_count;
+      if (p.out.n_runs) p.out.n_runs[e] = ec.run_count;
     }
   }
 }
@@ -420,6 +570,8 @@ cudaError_t kvs_launch_build(const BuildParams& p, int grid, cudaStream_t stream
   if (p.P <= 0) return cudaSuccess;
   cudaError_t err = cudaFuncSetAttribute(k_build_eval, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(build_smem_bytes()));
+  if (err != cudaSuccess) return err;
+  err = cudaMemsetAsync(p.counter, 0, 8, stream);   // work counter: CTAs draw evaluations from it
   if (err != cudaSuccess) return err;
   k_build_eval<<<grid, KVS_EVAL_THREADS, build_smem_bytes(), stream>>>(p);
   return cudaGetLastError();

@@ -50,6 +50,7 @@ struct BuildParams {
   int do_profile;
   // per-CTA carry lists: 2 * max_jobs entries each
   int32_t* lists;
+  ull* counter;             // next evaluation to hand out (zeroed before each launch)
 };
 
 struct SortParams {
