@@ -168,6 +168,7 @@ struct Acc {
 // Everything one phase needs that does not change while it runs.
 struct Phase {
   i64 base, tau, k, t_end;
+  i64 qt, rt;               // tau = qt * k + rt: the start offset advances by qt (+1 on carry) per rank
   int N, C, ent_lo, ph, seg_lo;
   bool simultaneous, geometric, may_carry, profile_on, combine;
 };
@@ -193,39 +194,60 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
   const int tid = threadIdx.x;
   u32* const dA = reinterpret_cast<u32*>(sh.dA);
   u32* const dB = reinterpret_cast<u32*>(sh.dB);
-  const i64 qt = P.tau / P.k, rt = P.tau % P.k;
-  for (i64 c0 = ra; c0 < rb; c0 += CHUNK) {
-    const i64 r_first = c0 + static_cast<i64>(tid) * RPT;
-    i64 q = 0, rem = 0;   // start offset of the current rank and the remainder that advances it
-    if (r_first < rb) {
-      if (P.simultaneous) { q = (r_first / P.k) * P.tau; rem = r_first % P.k; }
-      else {
-        const u64 x = static_cast<u64>(r_first) * static_cast<u64>(P.tau);
-        if ((x >> 32) == 0) { q = static_cast<u32>(x) / static_cast<u32>(P.k); rem = static_cast<u32>(x) % static_cast<u32>(P.k); }
-        else { q = static_cast<i64>(x / static_cast<u64>(P.k)); rem = static_cast<i64>(x % static_cast<u64>(P.k)); }
-      }
-    }
+  const i64 qt = P.qt, rt = P.rt;
+  for (i64 c0 = ra; c0 < rb;) {
+    // short ranges are spread one run per thread; long ones give each thread consecutive ranks
+    const i64 left = rb - c0;
+    const int rpt = left > 2 * T ? RPT : (left > T ? 2 : 1);
+    const i64 r_first = c0 + static_cast<i64>(tid) * rpt;
+    c0 += static_cast<i64>(T) * rpt;
     int cpos[RPT];
     u32 cmask = 0;
+    if (r_first - static_cast<i64>(lane_id()) * rpt < rb) {   // warps past the end of the range skip the visit
+    // gather first, all loads of a stage in flight together: position -> (o, s) -> job index
+    int pos_[RPT], o_[RPT], s_[RPT], orig_[RPT];
+#pragma unroll
+    for (int j = 0; j < RPT; ++j) {
+      const i64 r = r_first + j;
+      pos_[j] = (j < rpt && r < rb) ? (r < P.C ? cur[r] : P.ent_lo + static_cast<int>(r - P.C)) : -1;
+    }
+#pragma unroll
+    for (int j = 0; j < RPT; ++j) {
+      o_[j] = pos_[j] >= 0 ? __ldg(ec.O + P.seg_lo + pos_[j]) : 0;
+      s_[j] = pos_[j] >= 0 ? __ldg(ec.S + P.seg_lo + pos_[j]) : 0;
+    }
+#pragma unroll
+    for (int j = 0; j < RPT; ++j) {
+      const bool need = pos_[j] >= 0 && (o_[j] <= P.tau || !P.geometric || ec.want_runs);
+      orig_[j] = need ? (ec.PERM ? __ldg(ec.PERM + P.seg_lo + pos_[j]) : P.seg_lo + pos_[j]) : 0;
+    }
+    i64 q = 0, rem = 0;   // start offset of the current rank and the remainder that advances it
+    if (r_first < rb) {
+      u64 dq_, dr_;
+      divmod_u(P.simultaneous ? static_cast<u64>(r_first) : static_cast<u64>(r_first) * static_cast<u64>(P.tau),
+               static_cast<u64>(P.k), &dq_, &dr_);
+      q = static_cast<i64>(P.simultaneous ? dq_ * static_cast<u64>(P.tau) : dq_);
+      rem = static_cast<i64>(dr_);
+    }
 #pragma unroll
     for (int j = 0; j < RPT; ++j) {
       const i64 r = r_first + j;
       int sidx = -1, eidx = -1;
       u32 c = 0;
       cpos[j] = 0;
-      if (r < rb) {
-        const int pos = r < P.C ? cur[r] : P.ent_lo + static_cast<int>(r - P.C);
-        const int oi = ec.O[P.seg_lo + pos], si = ec.S[P.seg_lo + pos];
+      if (pos_[j] >= 0) {
+        const int pos = pos_[j];
+        const int oi = o_[j], si = s_[j];
         const i64 start = P.base + q;
         const i64 d = oi < P.tau ? oi : P.tau;
         const bool fin = oi <= P.tau;
         acc.steps += d;
         acc.hmax = max_i64(acc.hmax, start + d);
         if (fin || !P.geometric || ec.want_runs) {
-          const int orig = ec.PERM ? ec.PERM[P.seg_lo + pos] : P.seg_lo + pos;
+          const int orig = orig_[j];
           if (fin) {
             const i64 done = start + oi;
-            acc.flow += done - (ec.ARR ? ec.ARR[orig] : 0);
+            acc.flow += done - (ec.ARR ? __ldg(ec.ARR + orig) : 0);
             if (p.out.job_start) p.out.job_start[ec.job_out + orig] = static_cast<int32_t>(start);
             if (p.out.job_completion) p.out.job_completion[ec.job_out + orig] = static_cast<int32_t>(done);
             if (p.out.job_start64) p.out.job_start64[ec.job_out + orig] = start;
@@ -264,6 +286,7 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
         add_event(dA, dB, sidx, c, 1u, P.combine);
         add_event(dA, dB, eidx, 0u - c, 0xffffffffu, P.combine);
       }
+    }
     }
     if (P.may_carry) {
       int total;
@@ -484,7 +507,12 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         P.simultaneous = simultaneous; P.geometric = geometric;
         P.may_carry = geometric && (family == KVS_GSA || p.key != nullptr);
         P.combine = simultaneous ? P.k >= 4 : P.k >= 2 * P.tau;  // several runs per round: combine equal targets within a warp
-        const i64 len = (simultaneous ? ((N - 1) / P.k) * P.tau : slot_offset(N - 1, P.tau, P.k)) + P.tau;
+        {
+          u64 a_, b_;
+          divmod_u(static_cast<u64>(P.tau), static_cast<u64>(P.k), &a_, &b_);
+          P.qt = static_cast<i64>(a_); P.rt = static_cast<i64>(b_);
+        }
+        const i64 len = (simultaneous ? static_cast<i64>(ceil_div_u(N, P.k) - 1) * P.tau : slot_offset(N - 1, P.tau, P.k)) + P.tau;
         P.t_end = base + len;
         if (profile_on && min_i64(N, P.k + 1) * (static_cast<i64>(stats.s_max) + P.tau) >= (static_cast<i64>(1) << 32)) {
           profile_on = false;
@@ -504,12 +532,24 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
           u32 A_run = 0, B_run = 0;
           i64 r_next = 0;
           int buf = 0;
+          // Ranks that start before offset u: ceil(u*k/tau) (SPS) or ceil(u/tau)*k (SimS).  The tile
+          // ends advance by TILE, so the quotient and remainder of u*mult/tau are stepped, with one
+          // division pair per phase instead of one per tile.
+          const u64 mult = simultaneous ? 1 : static_cast<u64>(P.k);
+          const u64 utau = static_cast<u64>(P.tau);
+          const u64 v1 = static_cast<u64>(t0_first + TILE - base) * mult, dv = static_cast<u64>(TILE) * mult;
+          u64 cq, cr, dq, dr;
+          divmod_u(v1, utau, &cq, &cr);
+          divmod_u(dv, utau, &dq, &dr);
           for (i64 t0 = t0_first; t0 < P.t_end; t0 += TILE) {
             const int wlen = static_cast<int>(min_i64(TILE, P.t_end - t0));
-            const i64 u_hi = t0 + wlen - base;   // ranks starting before this offset belong to tiles up to this one
-            i64 r_b = simultaneous ? ceil_div_u(u_hi, P.tau) * P.k
-                                   : ceil_div_u(static_cast<u64>(u_hi) * static_cast<u64>(P.k), P.tau);
-            if (r_b > N) r_b = N;
+            i64 r_b = N;                         // the last tile takes every remaining rank
+            if (t0 + TILE < P.t_end) {
+              r_b = static_cast<i64>(cq + (cr > 0)) * (simultaneous ? P.k : 1);
+              if (r_b > N) r_b = N;
+            }
+            cq += dq; cr += dr;
+            if (cr >= utau) { cr -= utau; ++cq; }
             C_next = process_runs(p, sh, ec, P, cur, nxt, C_next, r_next, r_b, t0, buf, acc);
             r_next = r_b;
             if (P.tau > TILE) insert_far_ends(sh, ec, P, cur, t0_first, t0, wlen, buf);

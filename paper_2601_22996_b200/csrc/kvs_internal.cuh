@@ -117,7 +117,22 @@ __device__ __forceinline__ i64 slot_offset(i64 r, i64 tau, i64 k) {
   return static_cast<i64>(x / static_cast<u64>(k));
 }
 
-__device__ __forceinline__ i64 ceil_div_u(u64 x, u64 y) { return static_cast<i64>((x + y - 1) / y); }
+// Quotient and remainder of non-negative 64-bit values.  64-bit division is emulated with well over
+// a hundred instructions, so the common case of operands below 2^32 takes the 32-bit divider.
+__device__ __forceinline__ void divmod_u(u64 x, u64 y, u64* q, u64* r) {
+  if (((x | y) >> 32) == 0) {
+    const u32 a = static_cast<u32>(x), b = static_cast<u32>(y);
+    *q = a / b; *r = a % b;
+  } else {
+    *q = x / y; *r = x % y;
+  }
+}
+
+__device__ __forceinline__ i64 ceil_div_u(u64 x, u64 y) {
+  u64 q, r;
+  divmod_u(x, y, &q, &r);
+  return static_cast<i64>(q + (r != 0));
+}
 __device__ __forceinline__ i64 min_i64(i64 x, i64 y) { return x < y ? x : y; }
 __device__ __forceinline__ i64 max_i64(i64 x, i64 y) { return x > y ? x : y; }
 
