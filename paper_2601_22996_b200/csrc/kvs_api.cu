@@ -40,7 +40,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // one stream, so the entry points reuse the workspace from offset 0; the layout without staging
 // is a prefix of the layout with staging.
 struct Layout {
-  size_t settings, stats, perm, perm_tmp, sorted_s, sorted_o, sorted_key, lists, counter;
+  size_t settings, stats, perm, perm_tmp, sorted_s, sorted_o, sorted_key, prefix_s, lists, counter;
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -57,6 +57,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.sorted_s = take(static_cast<size_t>(N) * 4);
   L.sorted_o = take(static_cast<size_t>(N) * 4);
   L.sorted_key = take(static_cast<size_t>(N) * 4);
+  L.prefix_s = take(static_cast<size_t>(N + I) * 8);
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
   L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 4);
   L.counter = take(8);
@@ -195,6 +196,12 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   sp.sorted_s = reinterpret_cast<int32_t*>(ws + L.sorted_s);
   sp.sorted_o = reinterpret_cast<int32_t*>(ws + L.sorted_o);
   sp.sorted_key = reinterpret_cast<int32_t*>(ws + L.sorted_key);
+  // SPS / SimS evaluations that ask for no profile take the peak from run ends instead of rounds;
+  // that needs prefix sums of s in key order (exact keys only)
+  bool event_form = false;
+  if (do_profile && !inst->o_est)
+    for (int64_t e = 0; e < P && !event_form; ++e) event_form = settings[e].family >= KVS_SPS;
+  sp.prefix_s = event_form ? reinterpret_cast<i64*>(ws + L.prefix_s) : nullptr;
   const int64_t sort_cap = static_cast<int64_t>(ctx->sm_count) * 2;
   const int sort_grid = static_cast<int>(I < sort_cap ? I : sort_cap);
   if (ctx->timing) cudaEventRecord(ctx->ev[0], ctx->stream);
@@ -206,6 +213,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.job_off = inst->job_off; bp.s = inst->s; bp.o = inst->o; bp.key = inst->o_est; bp.arrival = inst->arrival;
   bp.window = inst->window; bp.n_instances = I; bp.max_jobs = max_n;
   bp.perm = sp.perm; bp.sorted_s = sp.sorted_s; bp.sorted_o = sp.sorted_o; bp.sorted_key = sp.sorted_key;
+  bp.prefix_s = sp.prefix_s;
   bp.stats = sp.stats;
   bp.settings = reinterpret_cast<const kvs_setting*>(ws + L.settings);
   bp.P = P; bp.out = o; bp.ev = v; bp.do_profile = do_profile;

@@ -23,7 +23,7 @@
 // The difference arrays and their sums are kept modulo 2^32.  Every intermediate may wrap, the
 // final memory(t) is exact whenever it is below 2^32, which a per-phase bound guarantees
 // (otherwise the evaluation reports KVS_EVAL_RANGE and skips the profile).
-#include "kvs_internal.cuh"
+#include "kvs_events.cuh"
 
 namespace {
 
@@ -162,7 +162,8 @@ __device__ __forceinline__ int block_count_scan(int v, int* red32, int* total) {
 struct Acc {
   i64 flow = 0, steps = 0, hmax = 0;
   int unfinished = 0;
-  u32 peak = 0;
+  u32 peak = 0;             // from the profile tiles
+  i64 peak64 = 0;           // from the event form
 };
 
 // Everything one phase needs that does not change while it runs.
@@ -514,15 +515,28 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         }
         const i64 len = (simultaneous ? static_cast<i64>(ceil_div_u(N, P.k) - 1) * P.tau : slot_offset(N - 1, P.tau, P.k)) + P.tau;
         P.t_end = base + len;
-        if (profile_on && min_i64(N, P.k + 1) * (static_cast<i64>(stats.s_max) + P.tau) >= (static_cast<i64>(1) << 32)) {
+        // SPS / SimS in exact key order with no profile wanted: the peak comes from the run ends
+        // (kvs_events.cuh), no rounds are walked
+        const bool event_form = profile_on && !geometric && p.prefix_s != nullptr && ec.prof_cap == 0;
+        if (profile_on && !event_form &&
+            min_i64(N, P.k + 1) * (static_cast<i64>(stats.s_max) + P.tau) >= (static_cast<i64>(1) << 32)) {
           profile_on = false;
           status |= KVS_EVAL_RANGE;
         }
-        P.profile_on = profile_on;
+        P.profile_on = profile_on && !event_form;
 
         int C_next = 0;
-        if (!profile_on) {
+        if (!P.profile_on) {
           C_next = process_runs(p, sh, ec, P, cur, nxt, 0, 0, N, 0, 0, acc);
+          if (event_form) {
+            const i64* const ps = p.prefix_s + lo + st.instance + seg_lo;
+            const i64 per = (static_cast<i64>(N) + T - 1) / T;
+            const i64 i0 = min_i64(N, tid * per), i1 = min_i64(N, i0 + per);
+            u64 unused_flow = 0;
+            const i64 pk = simultaneous ? sims_range_peak(ec.O + seg_lo, ps, N, P.tau, P.k, i0, i1, &unused_flow)
+                                        : sps_range_peak(ec.O + seg_lo, ps, N, P.tau, P.k, i0, i1, &unused_flow);
+            acc.peak64 = max_i64(acc.peak64, pk);
+          }
         } else {
           // idle rounds before this phase (window release) hold nothing
           if (ec.prof_cap > 0)
@@ -574,7 +588,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
     const i64 steps = block_sum(acc.steps, sh.red64);
     const i64 hmax = block_max(acc.hmax, sh.red64, static_cast<i64>(0));
     const int unfinished = block_sum(acc.unfinished, sh.red32);
-    const u32 peak = block_max(acc.peak, sh.redA, 0u);
+    const u32 peak32 = block_max(acc.peak, sh.redA, 0u);
+    const i64 peak = max_i64(static_cast<i64>(peak32), block_max(acc.peak64, sh.red64, static_cast<i64>(0)));
     if (tid == 0) {
       const bool skipped = (status & (KVS_EVAL_INFEASIBLE | KVS_EVAL_BAD_INPUT)) != 0;
       if (!skipped) {
@@ -583,12 +598,12 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         if (ec.prof_cap > 0 && hmax > ec.prof_cap) status |= KVS_EVAL_CAPACITY;   // capacity 0 = profile not wanted
       }
       const bool have_peak = p.do_profile && profile_on && !skipped;
-      if (p.ev.peak) p.ev.peak[e] = have_peak ? static_cast<i64>(peak) : -1;
+      if (p.ev.peak) p.ev.peak[e] = have_peak ? peak : -1;
       if (p.ev.flow) p.ev.flow[e] = flow;
       if (p.ev.job_steps) p.ev.job_steps[e] = steps;
       if (p.ev.horizon) p.ev.horizon[e] = hmax;
       if (p.ev.n_unfinished) p.ev.n_unfinished[e] = unfinished;
-      if (p.ev.feasible) p.ev.feasible[e] = (have_peak && !(status & KVS_EVAL_RANGE) && static_cast<i64>(peak) <= M) ? 1 : 0;
+      if (p.ev.feasible) p.ev.feasible[e] = (have_peak && !(status & KVS_EVAL_RANGE) && peak <= M) ? 1 : 0;
       if (p.ev.status) p.ev.status[e] = status;
       if (p.out.n_runs) p.out.n_runs[e] = ec.run_count;
     }

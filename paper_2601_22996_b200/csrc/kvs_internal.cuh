@@ -41,6 +41,7 @@ struct BuildParams {
   const int32_t* sorted_s;
   const int32_t* sorted_o;
   const int32_t* sorted_key;
+  const i64* prefix_s;      // see SortParams; NULL when no evaluation takes the event form of the peak
   const InstStats* stats;
   // evaluations
   const kvs_setting* settings;
@@ -69,6 +70,8 @@ struct SortParams {
   int32_t* sorted_s;
   int32_t* sorted_o;
   int32_t* sorted_key;      // written only when key != NULL
+  i64* prefix_s;            // NULL, or [n_jobs_total + n_instances]: instance j holds its n + 1 exclusive
+                            // prefix sums of s in schedule order at job_off[j] + j
 };
 
 struct GenericParams {

@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
   __shared__ u32 hist[4][256];
   __shared__ u32 bucket[256];
   __shared__ int red[32];
+  __shared__ i64 wsum[32];
   __shared__ int seg_end;
   const int tid = threadIdx.x;
 
@@ -147,6 +148,36 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       }
       __syncthreads();
       seg_lo = seg_hi;
+    }
+    if (p.prefix_s) {
+      // exclusive prefix sums of s in schedule order (n + 1 entries per instance): the event form
+      // of the peak reads the prompt tokens of any contiguous rank range as one difference
+      i64* const ps = p.prefix_s + lo + inst;
+      i64 run = 0;
+      if (tid == 0) ps[0] = 0;
+      for (int j0 = 0; j0 < n; j0 += T) {
+        const int j = j0 + tid;
+        const i64 v = j < n ? p.sorted_s[lo + j] : 0;
+        i64 incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const i64 y = __shfl_up_sync(0xffffffffu, incl, d);
+          if (static_cast<int>(lane_id()) >= d) incl += y;
+        }
+        __syncthreads();
+        if (lane_id() == 31) wsum[tid >> 5] = incl;
+        __syncthreads();
+        const i64 w = wsum[lane_id()];
+        i64 wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const i64 y = __shfl_up_sync(0xffffffffu, wi, d);
+          if (static_cast<int>(lane_id()) >= d) wi += y;
+        }
+        const i64 before = run + __shfl_sync(0xffffffffu, wi - w, tid >> 5);   // all lanes take part in the shuffle
+        if (j < n) ps[j + 1] = before + incl;
+        run += __shfl_sync(0xffffffffu, wi, 31);
+      }
     }
   }
 }

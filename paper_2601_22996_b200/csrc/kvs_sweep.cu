@@ -1,41 +1,14 @@
 // Parameter sweep: SPS or the simultaneous schedule for every (tau, k) of a grid on one
-// instance, scalars only.  Horizons reach billions of rounds, so nothing dense is formed.
-//
-// Jobs are in key order (key = exact response length), rank i starts at floor(i*tau/k)
-// (Procedure StaggeredPipelineSchedule) or floor(i/k)*tau (simultaneous batches) and runs
-// d_i = min(o_i, tau) rounds.  Starts and run lengths are both nondecreasing in i, hence so are
-// the run ends, and the jobs active in round t are a contiguous index range [e, b).  Memory is
-// piecewise linear and increasing between events, so its maximum is attained in the last round
-// of some run, t = end_i - 1, where
-//     memory(t) = sum_{j in [i, b)} (s_j + t - start_j + 1)
-//               = PS_s[b] - PS_s[i] + (b - i)(t + 1) - sum_{j in [i, b)} start_j
-// with b = #{j : start_j <= t} = min(n, ceil((t+1)k/tau))  (the count c(rho) in the proof of Lemma
-// "Peak Memory Usage of SPS").  Using i instead of the first index with the same end can only
-// drop non-negative terms, and that first index is itself a candidate, so the maximum is exact.
-// Each thread walks consecutive candidates, sliding the window sum of starts; long jumps of b use
-// the closed form sum_{j<n} floor(j*tau/k) (Euclid-like floor sum).
-#include "kvs_internal.cuh"
+// instance, scalars only.  Horizons reach billions of rounds, so nothing dense is formed: the
+// peak comes from the candidate rounds described in kvs_events.cuh, one CTA per (setting, chunk
+// of 8,192 ranks), each thread walking 64 consecutive ranks.
+#include "kvs_events.cuh"
 
 namespace {
 
 constexpr int SW_THREADS = 128;
 constexpr int SW_PER = 64;
 constexpr int SW_CHUNK = SW_THREADS * SW_PER;
-
-// sum_{j=0}^{n-1} floor((a*j + b) / m), arithmetic modulo 2^64
-__device__ u64 floor_sum(u64 n, u64 m, u64 a, u64 b) {
-  u64 ans = 0;
-  for (;;) {
-    if (a >= m) { ans += (n - 1) * n / 2 * (a / m); a %= m; }
-    if (b >= m) { ans += n * (b / m); b %= m; }
-    const u64 y = a * n + b;
-    if (y < m) break;
-    n = y / m;
-    b = y % m;
-    const u64 t = m; m = a; a = t;
-  }
-  return ans;
-}
 
 __global__ void __launch_bounds__(SW_THREADS) k_sweep(SweepParams p, i64 n_chunks, i64* acc_peak, u64* acc_flow) {
   __shared__ i64 red64[32];
@@ -44,56 +17,9 @@ __global__ void __launch_bounds__(SW_THREADS) k_sweep(SweepParams p, i64 n_chunk
   const i64 n = p.n;
   const i64 i0 = chunk * SW_CHUNK + static_cast<i64>(threadIdx.x) * SW_PER;
   const i64 i1 = i0 + SW_PER < n ? i0 + SW_PER : n;
-  i64 peak = 0;
   u64 flow = 0;
-  if (i0 < n) {
-    if (p.family == KVS_SPS) {
-      const i64 qt = tau / k, rt = tau % k;
-      u64 x = static_cast<u64>(i0) * static_cast<u64>(tau);
-      i64 qi = static_cast<i64>(x / static_cast<u64>(k)), ri = static_cast<i64>(x % static_cast<u64>(k));
-      i64 b = i0, qb = qi, rb = ri;   // b: first job not yet counted as started; (qb, rb): its start and remainder
-      u64 W = 0;                      // sum of starts over [i, b)
-      for (i64 i = i0; i < i1; ++i) {
-        const i64 oi = p.sorted_o[i];
-        const i64 d = oi < tau ? oi : tau;
-        const i64 t = qi + d - 1;     // last round of run i
-        if (oi <= tau) flow += static_cast<u64>(qi + oi);
-        int steps = 0;
-        while (b < n && qb <= t) {
-          if (steps == 32) {          // long jump: closed forms instead of stepping
-            i64 bn = ceil_div_u(static_cast<u64>(t + 1) * static_cast<u64>(k), static_cast<u64>(tau));
-            if (bn > n) bn = n;
-            W += floor_sum(bn, k, tau, 0) - floor_sum(b, k, tau, 0);
-            b = bn;
-            x = static_cast<u64>(b) * static_cast<u64>(tau);
-            qb = static_cast<i64>(x / static_cast<u64>(k)); rb = static_cast<i64>(x % static_cast<u64>(k));
-            break;
-          }
-          W += static_cast<u64>(qb);
-          ++b; rb += rt; qb += qt;
-          if (rb >= k) { rb -= k; ++qb; }
-          ++steps;
-        }
-        const i64 mem = (p.prefix_s[b] - p.prefix_s[i]) + (b - i) * (t + 1) - static_cast<i64>(W);
-        peak = mem > peak ? mem : peak;
-        W -= static_cast<u64>(qi);
-        ri += rt; qi += qt;
-        if (ri >= k) { ri -= k; ++qi; }
-      }
-    } else {
-      i64 j = i0 / k, rem = i0 % k;   // batch index and position inside the batch
-      for (i64 i = i0; i < i1; ++i) {
-        const i64 oi = p.sorted_o[i];
-        const i64 d = oi < tau ? oi : tau;
-        if (oi <= tau) flow += static_cast<u64>(j * tau + oi);
-        i64 bend = (j + 1) * k;
-        if (bend > n) bend = n;
-        const i64 mem = (p.prefix_s[bend] - p.prefix_s[i]) + (bend - i) * d;   // round start + d - 1 of the batch
-        peak = mem > peak ? mem : peak;
-        if (++rem == k) { rem = 0; ++j; }
-      }
-    }
-  }
+  i64 peak = p.family == KVS_SPS ? sps_range_peak(p.sorted_o, p.prefix_s, n, tau, k, i0, i1, &flow)
+                                 : sims_range_peak(p.sorted_o, p.prefix_s, n, tau, k, i0, i1, &flow);
   peak = block_max(peak, red64, static_cast<i64>(0));
   const i64 fsum = block_sum(static_cast<i64>(flow), red64);
   if (threadIdx.x == 0) {
