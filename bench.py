@@ -144,7 +144,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     name = args.workload
-    n_sample = 4 if name != "c3" else 1
+    n_sample = 32 if name != "c3" else 2
     inst = make_instances(name, n_sample, "cpu")
     settings, window = make_settings(name, inst)
     per = []
@@ -299,7 +299,7 @@ def run_ours(args):
     if e2e:
         line["e2e"] = {"value": steps_all / (e2e_s / args.steps), "unit": UNIT, "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2]}
     if not args.no_cpu:
-        n_s = 4 if name != "c3" else 1
+        n_s = 512 if name != "c3" else 8      # upper bound; the time budget ends the sample earlier
         cpu_inst = inst.slice(0, min(n_s, I)).to("cpu")
         cpu_inst.meta = dict(inst.meta)
         st, ev_n, dt = oracle_sample(name, cpu_inst, settings, window, args.cpu_seconds)
