@@ -40,7 +40,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // one stream, so the entry points reuse the workspace from offset 0; the layout without staging
 // is a prefix of the layout with staging.
 struct Layout {
-  size_t settings, stats, perm, perm_tmp, sorted_s, sorted_o, sorted_key, prefix_s, lists, counter;
+  size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter;
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -58,8 +58,10 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.sorted_o = take(static_cast<size_t>(N) * 4);
   L.sorted_key = take(static_cast<size_t>(N) * 4);
   L.prefix_s = take(static_cast<size_t>(N + I) * 8);
+  L.iperm = take(static_cast<size_t>(N) * 4);
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
   L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 4);
+  L.fin_rank = take(static_cast<size_t>(grid) * static_cast<size_t>(max_n) * 4);
   L.counter = take(8);
   if (staging) {
     L.st_off = take(static_cast<size_t>(I + 1) * 8);
@@ -193,6 +195,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
   sp.perm = reinterpret_cast<int32_t*>(ws + L.perm);
   sp.perm_tmp = reinterpret_cast<int32_t*>(ws + L.perm_tmp);
+  sp.iperm = reinterpret_cast<int32_t*>(ws + L.iperm);
   sp.sorted_s = reinterpret_cast<int32_t*>(ws + L.sorted_s);
   sp.sorted_o = reinterpret_cast<int32_t*>(ws + L.sorted_o);
   sp.sorted_key = reinterpret_cast<int32_t*>(ws + L.sorted_key);
@@ -214,6 +217,8 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.window = inst->window; bp.n_instances = I; bp.max_jobs = max_n;
   bp.perm = sp.perm; bp.sorted_s = sp.sorted_s; bp.sorted_o = sp.sorted_o; bp.sorted_key = sp.sorted_key;
   bp.prefix_s = sp.prefix_s;
+  bp.iperm = sp.iperm;
+  bp.fin_rank = reinterpret_cast<int32_t*>(ws + L.fin_rank);
   bp.stats = sp.stats;
   bp.settings = reinterpret_cast<const kvs_setting*>(ws + L.settings);
   bp.P = P; bp.out = o; bp.ev = v; bp.do_profile = do_profile;

@@ -61,6 +61,7 @@ struct Shared {
   uint4 dB[2][TILE / 4];    //                and of the slopes
   i64 tau[KVS_MAX_PHASES];
   i64 k[KVS_MAX_PHASES];
+  i64 pbase[KVS_MAX_PHASES];    // first round of each phase of the current window
   int ent[KVS_MAX_PHASES + 1];  // class boundaries in key order: entrants of phase p are [ent[p], ent[p+1])
   u128 pw_a[KVS_MAX_PHASES + 1];
   u128 pw_b[KVS_MAX_PHASES + 1];
@@ -180,6 +181,10 @@ struct EvalCtx {
   const int32_t* O;       // response lengths in schedule order
   const int32_t* PERM;    // schedule order -> job index inside the instance, or NULL (identity)
   const i64* ARR;         // arrivals of the instance, or NULL
+  const int32_t* O_JOB;   // response lengths in original job order
+  const int32_t* KEY_JOB; // estimates in original job order, or NULL (exact keys)
+  const int32_t* IPERM;   // job index -> position in schedule order, or NULL (identity)
+  int32_t* fin_rank;      // scratch of this CTA: rank of a job in the phase that completes it
   i64 job_out;            // offset of the evaluation's per-job block
   i64 run_base, run_cap, run_count;
   i64 prof_base, prof_cap;
@@ -219,7 +224,7 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
     }
 #pragma unroll
     for (int j = 0; j < RPT; ++j) {
-      const bool need = pos_[j] >= 0 && (o_[j] <= P.tau || !P.geometric || ec.want_runs);
+      const bool need = pos_[j] >= 0 && ec.want_runs;   // only the explicit run list names the job
       orig_[j] = need ? (ec.PERM ? __ldg(ec.PERM + P.seg_lo + pos_[j]) : P.seg_lo + pos_[j]) : 0;
     }
     i64 q = 0, rem = 0;   // start offset of the current rank and the remainder that advances it
@@ -244,30 +249,16 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
         const bool fin = oi <= P.tau;
         acc.steps += d;
         acc.hmax = max_i64(acc.hmax, start + d);
-        if (fin || !P.geometric || ec.want_runs) {
-          const int orig = orig_[j];
-          if (fin) {
-            const i64 done = start + oi;
-            acc.flow += done - (ec.ARR ? __ldg(ec.ARR + orig) : 0);
-            if (p.out.job_start) p.out.job_start[ec.job_out + orig] = static_cast<int32_t>(start);
-            if (p.out.job_completion) p.out.job_completion[ec.job_out + orig] = static_cast<int32_t>(done);
-            if (p.out.job_start64) p.out.job_start64[ec.job_out + orig] = start;
-            if (p.out.job_completion64) p.out.job_completion64[ec.job_out + orig] = done;
-          } else if (!P.geometric) {
-            ++acc.unfinished;
-            if (p.out.job_start) p.out.job_start[ec.job_out + orig] = -1;
-            if (p.out.job_completion) p.out.job_completion[ec.job_out + orig] = -1;
-            if (p.out.job_start64) p.out.job_start64[ec.job_out + orig] = -1;
-            if (p.out.job_completion64) p.out.job_completion64[ec.job_out + orig] = -1;
-          }
-          if (ec.want_runs && ec.run_count + r < ec.run_cap) {
-            const i64 w = ec.run_base + ec.run_count + r;
-            if (p.out.run_job) p.out.run_job[w] = orig;
-            if (p.out.run_phase) p.out.run_phase[w] = P.ph;
-            if (p.out.run_start) p.out.run_start[w] = start;
-            if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
-            if (p.out.run_s) p.out.run_s[w] = si;
-          }
+        // Per-job results are written later, in original job order (write_jobs); a job that
+        // completes among carried ones leaves its rank for that pass.
+        if (fin && P.may_carry) ec.fin_rank[P.seg_lo + pos] = static_cast<int32_t>(r);
+        if (ec.want_runs && ec.run_count + r < ec.run_cap) {
+          const i64 w = ec.run_base + ec.run_count + r;
+          if (p.out.run_job) p.out.run_job[w] = orig_[j];
+          if (p.out.run_phase) p.out.run_phase[w] = P.ph;
+          if (p.out.run_start) p.out.run_start[w] = start;
+          if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
+          if (p.out.run_s) p.out.run_s[w] = si;
         }
         if (!fin && P.geometric) { cpos[j] = pos; cmask |= 1u << j; }
         if (P.profile_on) {
@@ -394,6 +385,49 @@ __device__ __forceinline__ void insert_far_ends(Shared& sh, const EvalCtx& ec, c
   }
 }
 
+// Per-job results of one window, written in original job order so that the stores are contiguous.
+// The phase that completes job j is the later of its key's class and the class of o_j
+// (class(x) = first p with tau_p >= x); its rank there is its position inside the class when no
+// jobs are carried, else the rank noted when it completed.  Also accumulates the flow time.
+__device__ __forceinline__ void write_jobs(const BuildParams& p, const Shared& sh, const EvalCtx& ec, int family,
+                                           int L, i64 X, int seg_lo, int seg_hi, bool may_carry, Acc& acc) {
+  const bool geometric = family == KVS_GBA || family == KVS_GSA;
+  const bool simultaneous = family == KVS_SIMS;
+  for (int j = seg_lo + threadIdx.x; j < seg_hi; j += T) {
+    const int oj = __ldg(ec.O_JOB + j);
+    const int pos = ec.IPERM ? __ldg(ec.IPERM + j) : j;
+    int ph = 0;
+    bool fin = true;
+    if (geometric) {
+      i64 x = oj;
+      if (family == KVS_GBA && ec.KEY_JOB) {          // class of the estimate, clipped to [1, X]
+        i64 kj = __ldg(ec.KEY_JOB + j);
+        kj = kj < 1 ? 1 : (kj > X ? X : kj);
+        x = kj > x ? kj : x;                          // classes are monotone: max of classes = class of max
+      }
+      int a = 0, b = L - 1;                           // tau_(L-1) = X >= x
+      while (a < b) { const int m = (a + b) >> 1; if (sh.tau[m] >= x) b = m; else a = m + 1; }
+      ph = a;
+    } else {
+      fin = oj <= sh.tau[0];
+    }
+    i64 start = -1, done = -1;
+    if (fin) {
+      const i64 rank = may_carry ? static_cast<i64>(ec.fin_rank[pos]) : static_cast<i64>(pos - seg_lo - sh.ent[ph]);
+      const i64 tau = sh.tau[ph], k = sh.k[ph];
+      start = sh.pbase[ph] + (simultaneous ? (rank / k) * tau : slot_offset(rank, tau, k));
+      done = start + oj;
+      acc.flow += done - (ec.ARR ? __ldg(ec.ARR + j) : 0);
+    } else {
+      ++acc.unfinished;
+    }
+    if (p.out.job_start) p.out.job_start[ec.job_out + j] = static_cast<int32_t>(start);
+    if (p.out.job_completion) p.out.job_completion[ec.job_out + j] = static_cast<int32_t>(done);
+    if (p.out.job_start64) p.out.job_start64[ec.job_out + j] = start;
+    if (p.out.job_completion64) p.out.job_completion64[ec.job_out + j] = done;
+  }
+}
+
 __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
@@ -429,6 +463,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
     ec.O = (keyed ? p.sorted_o : p.o) + lo;
     ec.PERM = keyed ? p.perm + lo : nullptr;
     ec.ARR = p.arrival ? p.arrival + lo : nullptr;
+    ec.O_JOB = p.o + lo;
+    ec.KEY_JOB = p.key ? p.key + lo : nullptr;
+    ec.IPERM = keyed ? p.iperm + lo : nullptr;
+    ec.fin_rank = p.fin_rank + static_cast<i64>(blockIdx.x) * p.max_jobs;
     ec.job_out = p.out.job_out_off ? p.out.job_out_off[e] : 0;
     ec.run_base = p.out.run_off ? p.out.run_off[e] : 0;
     ec.run_cap = p.out.run_off ? p.out.run_off[e + 1] - ec.run_base : 0;
@@ -503,6 +541,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         const int N = C + (ent_hi - ent_lo);
         if (N == 0) continue;          // an empty class takes no time
         Phase P;
+        if (tid == 0) sh.pbase[ph] = base;   // read by write_jobs after the window's last barrier
         P.base = base; P.tau = sh.tau[ph]; P.k = sh.k[ph];
         P.N = N; P.C = C; P.ent_lo = ent_lo; P.ph = ph; P.seg_lo = seg_lo;
         P.simultaneous = simultaneous; P.geometric = geometric;
@@ -580,6 +619,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         C = C_next;
         if (C == 0 && ent_hi == nseg) break;   // nothing left in this window
       }
+      write_jobs(p, sh, ec, family, L, X, seg_lo, seg_hi, geometric && (family == KVS_GSA || p.key != nullptr), acc);
       seg_lo = seg_hi;
     }
 

@@ -42,6 +42,8 @@ struct BuildParams {
   const int32_t* sorted_o;
   const int32_t* sorted_key;
   const i64* prefix_s;      // see SortParams; NULL when no evaluation takes the event form of the peak
+  const int32_t* iperm;     // job index inside the instance -> position in key order
+  int32_t* fin_rank;        // per-CTA scratch, max_jobs entries each
   const InstStats* stats;
   // evaluations
   const kvs_setting* settings;
@@ -67,6 +69,7 @@ struct SortParams {
   InstStats* stats;
   int32_t* perm;
   int32_t* perm_tmp;
+  int32_t* iperm;           // inverse of perm (job index -> position), or NULL
   int32_t* sorted_s;
   int32_t* sorted_o;
   int32_t* sorted_key;      // written only when key != NULL

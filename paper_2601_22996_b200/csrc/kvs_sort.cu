@@ -145,6 +145,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
         p.sorted_s[lo + j] = p.s[lo + idx];
         p.sorted_o[lo + j] = p.o[lo + idx];
         if (p.key) p.sorted_key[lo + j] = p.key[lo + idx];
+        if (p.iperm) p.iperm[lo + idx] = j;
       }
       __syncthreads();
       seg_lo = seg_hi;
