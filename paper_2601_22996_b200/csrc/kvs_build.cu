@@ -194,7 +194,8 @@ struct EvalCtx {
 // Visits ranks [ra, rb) of a phase once: outputs, carry list, and (if the profile is on) the two
 // events of every run.  All of these runs start inside the tile with origin t0; `buf` is the ring
 // half of that tile.  Returns the new length of the carry list.
-__device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
+template <bool SIM, bool CARRY, bool EVENTS, bool RUNS>
+__device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
                                             const int32_t* cur, int32_t* nxt, int C_next, i64 ra, i64 rb,
                                             i64 t0, int buf, Acc& acc) {
   const int tid = threadIdx.x;
@@ -224,15 +225,15 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
     }
 #pragma unroll
     for (int j = 0; j < RPT; ++j) {
-      const bool need = pos_[j] >= 0 && ec.want_runs;   // only the explicit run list names the job
+      const bool need = pos_[j] >= 0 && RUNS;   // only the explicit run list names the job
       orig_[j] = need ? (ec.PERM ? __ldg(ec.PERM + P.seg_lo + pos_[j]) : P.seg_lo + pos_[j]) : 0;
     }
     i64 q = 0, rem = 0;   // start offset of the current rank and the remainder that advances it
     if (r_first < rb) {
       u64 dq_, dr_;
-      divmod_u(P.simultaneous ? static_cast<u64>(r_first) : static_cast<u64>(r_first) * static_cast<u64>(P.tau),
+      divmod_u(SIM ? static_cast<u64>(r_first) : static_cast<u64>(r_first) * static_cast<u64>(P.tau),
                static_cast<u64>(P.k), &dq_, &dr_);
-      q = static_cast<i64>(P.simultaneous ? dq_ * static_cast<u64>(P.tau) : dq_);
+      q = static_cast<i64>(SIM ? dq_ * static_cast<u64>(P.tau) : dq_);
       rem = static_cast<i64>(dr_);
     }
 #pragma unroll
@@ -251,8 +252,8 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
         acc.hmax = max_i64(acc.hmax, start + d);
         // Per-job results are written later, in original job order (write_jobs); a job that
         // completes among carried ones leaves its rank for that pass.
-        if (fin && P.may_carry) ec.fin_rank[P.seg_lo + pos] = static_cast<int32_t>(r);
-        if (ec.want_runs && ec.run_count + r < ec.run_cap) {
+        if (fin && CARRY) ec.fin_rank[P.seg_lo + pos] = static_cast<int32_t>(r);
+        if (RUNS && ec.run_count + r < ec.run_cap) {
           const i64 w = ec.run_base + ec.run_count + r;
           if (p.out.run_job) p.out.run_job[w] = orig_[j];
           if (p.out.run_phase) p.out.run_phase[w] = P.ph;
@@ -260,8 +261,8 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
           if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
           if (p.out.run_s) p.out.run_s[w] = si;
         }
-        if (!fin && P.geometric) { cpos[j] = pos; cmask |= 1u << j; }
-        if (P.profile_on) {
+        if (CARRY && !fin) { cpos[j] = pos; cmask |= 1u << j; }
+        if (EVENTS) {
           c = static_cast<u32>(si + 1) - static_cast<u32>(start);   // tokens(t) = c + t while active
           const int srel = static_cast<int>(start - t0);
           sidx = buf * TILE + slot(srel);
@@ -271,16 +272,16 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
             else if (erel < 2 * TILE) eidx = (buf ^ 1) * TILE + slot(static_cast<int>(erel - TILE));
           }
         }
-        if (P.simultaneous) { if (++rem == P.k) { rem = 0; q += P.tau; } }
+        if (SIM) { if (++rem == P.k) { rem = 0; q += P.tau; } }
         else { rem += rt; q += qt; if (rem >= P.k) { rem -= P.k; ++q; } }
       }
-      if (P.profile_on) {
+      if (EVENTS) {
         add_event(dA, dB, sidx, c, 1u, P.combine);
         add_event(dA, dB, eidx, 0u - c, 0xffffffffu, P.combine);
       }
     }
     }
-    if (P.may_carry) {
+    if (CARRY) {
       int total;
       int off = C_next + block_count_scan(__popc(cmask), sh.red32, &total);
 #pragma unroll
@@ -290,6 +291,22 @@ __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, co
     }
   }
   return C_next;
+}
+
+// Picks the specialisation: simultaneous starts, carried jobs, events and the explicit run list are
+// compile-time switches, so each variant carries only the registers and branches it needs.
+template <bool EVENTS>
+__device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
+                                            const int32_t* cur, int32_t* nxt, int C_next, i64 ra, i64 rb,
+                                            i64 t0, int buf, Acc& acc) {
+  if (ec.want_runs) {
+    if (P.simultaneous) return process_runs_t<true, false, EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+    if (P.may_carry) return process_runs_t<false, true, EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+    return process_runs_t<false, false, EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  }
+  if (P.simultaneous) return process_runs_t<true, false, EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  if (P.may_carry) return process_runs_t<false, true, EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  return process_runs_t<false, false, EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
 }
 
 // Prefix-sums one tile of the ring, turns it into memory(t), reduces the peak, stores the profile
@@ -566,7 +583,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
 
         int C_next = 0;
         if (!P.profile_on) {
-          C_next = process_runs(p, sh, ec, P, cur, nxt, 0, 0, N, 0, 0, acc);
+          C_next = process_runs<false>(p, sh, ec, P, cur, nxt, 0, 0, N, 0, 0, acc);
           if (event_form) {
             const i64* const ps = p.prefix_s + lo + st.instance + seg_lo;
             const i64 per = (static_cast<i64>(N) + T - 1) / T;
@@ -603,7 +620,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
             }
             cq += dq; cr += dr;
             if (cr >= utau) { cr -= utau; ++cq; }
-            C_next = process_runs(p, sh, ec, P, cur, nxt, C_next, r_next, r_b, t0, buf, acc);
+            C_next = process_runs<true>(p, sh, ec, P, cur, nxt, C_next, r_next, r_b, t0, buf, acc);
             r_next = r_b;
             if (P.tau > TILE) insert_far_ends(sh, ec, P, cur, t0_first, t0, wlen, buf);
             __syncthreads();
