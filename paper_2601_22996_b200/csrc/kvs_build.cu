@@ -563,7 +563,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         P.N = N; P.C = C; P.ent_lo = ent_lo; P.ph = ph; P.seg_lo = seg_lo;
         P.simultaneous = simultaneous; P.geometric = geometric;
         P.may_carry = geometric && (family == KVS_GSA || p.key != nullptr);
-        P.combine = simultaneous ? P.k >= 4 : P.k >= 2 * P.tau;  // several runs per round: combine equal targets within a warp
+        // Combining equal targets inside a warp (match + reduce) costs more than the serialised
+        // shared-memory atomics it saves unless a whole warp hits one word: only whole simultaneous
+        // batches do that.
+        P.combine = simultaneous && P.k >= 32;
         {
           u64 a_, b_;
           divmod_u(static_cast<u64>(P.tau), static_cast<u64>(P.k), &a_, &b_);
