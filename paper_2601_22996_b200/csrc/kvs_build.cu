@@ -194,92 +194,111 @@ struct EvalCtx {
 // Visits ranks [ra, rb) of a phase once: outputs, carry list, and (if the profile is on) the two
 // events of every run.  All of these runs start inside the tile with origin t0; `buf` is the ring
 // half of that tile.  Returns the new length of the carry list.
-template <bool SIM, bool CARRY, bool EVENTS, bool RUNS>
+template <bool WIDE> struct OffsetType { typedef int type; };
+template <> struct OffsetType<true> { typedef i64 type; };
+
+// SIM, CARRY, EVENTS, RUNS: simultaneous starts, carried jobs possible, events wanted, explicit run
+// list wanted.  WIDE: the phase is 2^30 rounds or longer, offsets inside it need 64 bits; otherwise
+// all per-run arithmetic is 32-bit (ranks, slice lengths and parallelism are below 2^31).
+template <bool SIM, bool CARRY, bool EVENTS, bool RUNS, bool WIDE>
 __device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
-                                            const int32_t* cur, int32_t* nxt, int C_next, i64 ra, i64 rb,
-                                            i64 t0, int buf, Acc& acc) {
+                                              const int32_t* cur, int32_t* nxt, int C_next, int ra, int rb,
+                                              i64 t0, int buf, Acc& acc) {
+  typedef typename OffsetType<WIDE>::type off_t;
   const int tid = threadIdx.x;
   u32* const dA = reinterpret_cast<u32*>(sh.dA);
   u32* const dB = reinterpret_cast<u32*>(sh.dB);
-  const i64 qt = P.qt, rt = P.rt;
-  for (i64 c0 = ra; c0 < rb;) {
+  const u32 tau = static_cast<u32>(P.tau), k = static_cast<u32>(P.k);
+  const u32 qt = static_cast<u32>(P.qt), rt = static_cast<u32>(P.rt);
+  const off_t trel = static_cast<off_t>(t0 - P.base);        // tile origin relative to the phase
+  const off_t len = static_cast<off_t>(P.t_end - P.base);
+  const u32 cbase = static_cast<u32>(P.base);
+  off_t far = 0;                                             // largest run end seen, relative to the phase
+  for (int c0 = ra; c0 < rb;) {
     // short ranges are spread one run per thread; long ones give each thread consecutive ranks
-    const i64 left = rb - c0;
+    const int left = rb - c0;
     const int rpt = left > 2 * T ? RPT : (left > T ? 2 : 1);
-    const i64 r_first = c0 + static_cast<i64>(tid) * rpt;
-    c0 += static_cast<i64>(T) * rpt;
+    const int r_first = c0 + tid * rpt;
+    c0 += T * rpt;
     int cpos[RPT];
     u32 cmask = 0;
-    if (r_first - static_cast<i64>(lane_id()) * rpt < rb) {   // warps past the end of the range skip the visit
-    // gather first, all loads of a stage in flight together: position -> (o, s) -> job index
-    int pos_[RPT], o_[RPT], s_[RPT], orig_[RPT];
+    if (r_first - static_cast<int>(lane_id()) * rpt < rb) {   // warps past the end of the range skip the visit
+      // gather first, all loads of a stage in flight together: position -> (o, s) -> job index
+      int pos_[RPT], o_[RPT], s_[RPT], orig_[RPT];
 #pragma unroll
-    for (int j = 0; j < RPT; ++j) {
-      const i64 r = r_first + j;
-      pos_[j] = (j < rpt && r < rb) ? (r < P.C ? cur[r] : P.ent_lo + static_cast<int>(r - P.C)) : -1;
-    }
+      for (int j = 0; j < RPT; ++j) {
+        const int r = r_first + j;
+        pos_[j] = (j < rpt && r < rb) ? (r < P.C ? cur[r] : P.ent_lo + (r - P.C)) : -1;
+      }
 #pragma unroll
-    for (int j = 0; j < RPT; ++j) {
-      o_[j] = pos_[j] >= 0 ? __ldg(ec.O + P.seg_lo + pos_[j]) : 0;
-      s_[j] = pos_[j] >= 0 ? __ldg(ec.S + P.seg_lo + pos_[j]) : 0;
-    }
+      for (int j = 0; j < RPT; ++j) {
+        o_[j] = pos_[j] >= 0 ? __ldg(ec.O + P.seg_lo + pos_[j]) : 0;
+        s_[j] = pos_[j] >= 0 ? __ldg(ec.S + P.seg_lo + pos_[j]) : 0;
+      }
+      if (RUNS) {
 #pragma unroll
-    for (int j = 0; j < RPT; ++j) {
-      const bool need = pos_[j] >= 0 && RUNS;   // only the explicit run list names the job
-      orig_[j] = need ? (ec.PERM ? __ldg(ec.PERM + P.seg_lo + pos_[j]) : P.seg_lo + pos_[j]) : 0;
-    }
-    i64 q = 0, rem = 0;   // start offset of the current rank and the remainder that advances it
-    if (r_first < rb) {
-      u64 dq_, dr_;
-      divmod_u(SIM ? static_cast<u64>(r_first) : static_cast<u64>(r_first) * static_cast<u64>(P.tau),
-               static_cast<u64>(P.k), &dq_, &dr_);
-      q = static_cast<i64>(SIM ? dq_ * static_cast<u64>(P.tau) : dq_);
-      rem = static_cast<i64>(dr_);
-    }
-#pragma unroll
-    for (int j = 0; j < RPT; ++j) {
-      const i64 r = r_first + j;
-      int sidx = -1, eidx = -1;
-      u32 c = 0;
-      cpos[j] = 0;
-      if (pos_[j] >= 0) {
-        const int pos = pos_[j];
-        const int oi = o_[j], si = s_[j];
-        const i64 start = P.base + q;
-        const i64 d = oi < P.tau ? oi : P.tau;
-        const bool fin = oi <= P.tau;
-        acc.steps += d;
-        acc.hmax = max_i64(acc.hmax, start + d);
-        // Per-job results are written later, in original job order (write_jobs); a job that
-        // completes among carried ones leaves its rank for that pass.
-        if (fin && CARRY) ec.fin_rank[P.seg_lo + pos] = static_cast<int32_t>(r);
-        if (RUNS && ec.run_count + r < ec.run_cap) {
-          const i64 w = ec.run_base + ec.run_count + r;
-          if (p.out.run_job) p.out.run_job[w] = orig_[j];
-          if (p.out.run_phase) p.out.run_phase[w] = P.ph;
-          if (p.out.run_start) p.out.run_start[w] = start;
-          if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
-          if (p.out.run_s) p.out.run_s[w] = si;
+        for (int j = 0; j < RPT; ++j)   // only the explicit run list names the job
+          orig_[j] = pos_[j] >= 0 ? (ec.PERM ? __ldg(ec.PERM + P.seg_lo + pos_[j]) : P.seg_lo + pos_[j]) : 0;
+      }
+      off_t q = 0;      // start offset of the current rank inside the phase
+      u32 rem = 0;      // and the remainder that advances it
+      if (r_first < rb) {
+        if (SIM) {
+          const u32 b = static_cast<u32>(r_first) / k;
+          q = static_cast<off_t>(b) * static_cast<off_t>(tau);
+          rem = static_cast<u32>(r_first) - b * k;
+        } else {
+          u64 dq_, dr_;
+          divmod_u(static_cast<u64>(r_first) * tau, k, &dq_, &dr_);
+          q = static_cast<off_t>(dq_);
+          rem = static_cast<u32>(dr_);
         }
-        if (CARRY && !fin) { cpos[j] = pos; cmask |= 1u << j; }
-        if (EVENTS) {
-          c = static_cast<u32>(si + 1) - static_cast<u32>(start);   // tokens(t) = c + t while active
-          const int srel = static_cast<int>(start - t0);
-          sidx = buf * TILE + slot(srel);
-          if (start + d < P.t_end) {                                  // an end at the phase end is never read
-            const i64 erel = srel + d;
-            if (erel < TILE) eidx = buf * TILE + slot(static_cast<int>(erel));
-            else if (erel < 2 * TILE) eidx = (buf ^ 1) * TILE + slot(static_cast<int>(erel - TILE));
+      }
+      u32 steps = 0;
+#pragma unroll
+      for (int j = 0; j < RPT; ++j) {
+        int sidx = -1, eidx = -1;
+        u32 c = 0;
+        cpos[j] = 0;
+        if (pos_[j] >= 0) {
+          const int r = r_first + j;
+          const u32 oi = static_cast<u32>(o_[j]);
+          const u32 d = oi < tau ? oi : tau;
+          const bool fin = oi <= tau;
+          const off_t end = q + static_cast<off_t>(d);
+          steps += d;
+          far = end > far ? end : far;
+          // Per-job results are written later, in original job order (write_jobs); a job that
+          // completes among carried ones leaves its rank for that pass.
+          if (CARRY && fin) ec.fin_rank[P.seg_lo + pos_[j]] = r;
+          if (RUNS && ec.run_count + r < ec.run_cap) {
+            const i64 w = ec.run_base + ec.run_count + r;
+            if (p.out.run_job) p.out.run_job[w] = orig_[j];
+            if (p.out.run_phase) p.out.run_phase[w] = P.ph;
+            if (p.out.run_start) p.out.run_start[w] = P.base + q;
+            if (p.out.run_len) p.out.run_len[w] = static_cast<int32_t>(d);
+            if (p.out.run_s) p.out.run_s[w] = s_[j];
           }
+          if (CARRY && !fin) { cpos[j] = pos_[j]; cmask |= 1u << j; }
+          if (EVENTS) {
+            c = static_cast<u32>(s_[j] + 1) - cbase - static_cast<u32>(q);   // tokens(t) = c + t while active
+            const int srel = static_cast<int>(q - trel);
+            sidx = buf * TILE + slot(srel);
+            if (end < len) {                                   // an end at the phase end is never read
+              const u32 erel = static_cast<u32>(srel) + d;
+              if (erel < TILE) eidx = buf * TILE + slot(static_cast<int>(erel));
+              else if (erel < 2 * TILE) eidx = (buf ^ 1) * TILE + slot(static_cast<int>(erel - TILE));
+            }
+          }
+          if (SIM) { if (++rem == k) { rem = 0; q += static_cast<off_t>(tau); } }
+          else { rem += rt; q += static_cast<off_t>(qt); if (rem >= k) { rem -= k; ++q; } }
         }
-        if (SIM) { if (++rem == P.k) { rem = 0; q += P.tau; } }
-        else { rem += rt; q += qt; if (rem >= P.k) { rem -= P.k; ++q; } }
+        if (EVENTS) {
+          add_event(dA, dB, sidx, c, 1u, P.combine);
+          add_event(dA, dB, eidx, 0u - c, 0xffffffffu, P.combine);
+        }
       }
-      if (EVENTS) {
-        add_event(dA, dB, sidx, c, 1u, P.combine);
-        add_event(dA, dB, eidx, 0u - c, 0xffffffffu, P.combine);
-      }
-    }
+      acc.steps += steps;
     }
     if (CARRY) {
       int total;
@@ -290,23 +309,33 @@ __device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, 
       C_next += total;
     }
   }
+  acc.hmax = max_i64(acc.hmax, P.base + static_cast<i64>(far));
   return C_next;
 }
 
-// Picks the specialisation: simultaneous starts, carried jobs, events and the explicit run list are
-// compile-time switches, so each variant carries only the registers and branches it needs.
+// Picks the specialisation: each variant carries only the registers and branches it needs.
+template <bool EVENTS, bool WIDE>
+__device__ __forceinline__ int process_runs_w(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
+                                              const int32_t* cur, int32_t* nxt, int C_next, int ra, int rb,
+                                              i64 t0, int buf, Acc& acc) {
+  if (ec.want_runs) {
+    if (P.simultaneous) return process_runs_t<true, false, EVENTS, true, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+    if (P.may_carry) return process_runs_t<false, true, EVENTS, true, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+    return process_runs_t<false, false, EVENTS, true, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  }
+  if (P.simultaneous) return process_runs_t<true, false, EVENTS, false, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  if (P.may_carry) return process_runs_t<false, true, EVENTS, false, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  return process_runs_t<false, false, EVENTS, false, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+}
+
 template <bool EVENTS>
 __device__ __forceinline__ int process_runs(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
                                             const int32_t* cur, int32_t* nxt, int C_next, i64 ra, i64 rb,
                                             i64 t0, int buf, Acc& acc) {
-  if (ec.want_runs) {
-    if (P.simultaneous) return process_runs_t<true, false, EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
-    if (P.may_carry) return process_runs_t<false, true, EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
-    return process_runs_t<false, false, EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
-  }
-  if (P.simultaneous) return process_runs_t<true, false, EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
-  if (P.may_carry) return process_runs_t<false, true, EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
-  return process_runs_t<false, false, EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  const int a = static_cast<int>(ra), b = static_cast<int>(rb);
+  if (P.t_end - P.base >= (static_cast<i64>(1) << 30))
+    return process_runs_w<EVENTS, true>(p, sh, ec, P, cur, nxt, C_next, a, b, t0, buf, acc);
+  return process_runs_w<EVENTS, false>(p, sh, ec, P, cur, nxt, C_next, a, b, t0, buf, acc);
 }
 
 // Prefix-sums one tile of the ring, turns it into memory(t), reduces the peak, stores the profile
