@@ -213,7 +213,7 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
   i64 X = M - s_bar;                      // largest response length that fits (per-job feasibility)
   if (X < 1) { S->status = 1; return S; }
   for (i64 i = 0; i < n; ++i) {
-    if (o[i] < 1 || s[i] < 0) { S->status = 3; return S; }
+    if (o[i] < 1 || s[i] < 0 || (o_est && o_est[i] < 1)) { S->status = 3; return S; }
     if (o[i] > X) { S->status = 1; return S; }
   }
   if (arrival)
