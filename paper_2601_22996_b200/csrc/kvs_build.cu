@@ -173,6 +173,7 @@ struct Phase {
   i64 qt, rt;               // tau = qt * k + rt: the start offset advances by qt (+1 on carry) per rank
   int N, C, ent_lo, ph, seg_lo;
   bool simultaneous, geometric, may_carry, profile_on, combine;
+  bool dense;               // several runs start per round and tau < TILE: events are combined per round
 };
 
 // Per-evaluation pointers and output windows.
@@ -255,6 +256,15 @@ __device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, 
         }
       }
       u32 steps = 0;
+      // Dense phases (several runs start per round): the runs of a lane that start in the round of
+      // its first run are summed in registers, then equal rounds - contiguous lanes, because
+      // consecutive ranks start in nondecreasing rounds - are summed across the warp with a
+      // segmented scan, and one lane per round issues the atomics.  Runs that hold their whole
+      // slot end together (start + tau), so their end events are combined the same way.
+      const bool dense = EVENTS && !SIM && P.dense;
+      int seg = 0x7fffffff;                 // round (relative to the tile) of the lane's segment
+      u32 seg_all = 0, seg_full = 0;        // sums of c over the segment: all runs / runs holding the whole slot
+      u32 seg_cnt = 0;                      // counts: all | full << 16
 #pragma unroll
       for (int j = 0; j < RPT; ++j) {
         int sidx = -1, eidx = -1;
@@ -266,8 +276,10 @@ __device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, 
           const u32 d = oi < tau ? oi : tau;
           const bool fin = oi <= tau;
           const off_t end = q + static_cast<off_t>(d);
-          steps += d;
-          far = end > far ? end : far;
+          if (CARRY) {   // without carried jobs there is one run per job, accounted in write_jobs
+            steps += d;
+            far = end > far ? end : far;
+          }
           // Per-job results are written later, in original job order (write_jobs); a job that
           // completes among carried ones leaves its rank for that pass.
           if (CARRY && fin) ec.fin_rank[P.seg_lo + pos_[j]] = r;
@@ -289,6 +301,14 @@ __device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, 
               if (erel < TILE) eidx = buf * TILE + slot(static_cast<int>(erel));
               else if (erel < 2 * TILE) eidx = (buf ^ 1) * TILE + slot(static_cast<int>(erel - TILE));
             }
+            if (dense) {
+              if (seg == 0x7fffffff) seg = srel;
+              if (srel == seg) {
+                seg_all += c; seg_cnt += 1u;
+                sidx = -1;
+                if (d == tau) { seg_full += c; seg_cnt += 1u << 16; eidx = -1; }
+              }
+            }
           }
           if (SIM) { if (++rem == k) { rem = 0; q += static_cast<off_t>(tau); } }
           else { rem += rt; q += static_cast<off_t>(qt); if (rem >= k) { rem -= k; ++q; } }
@@ -296,6 +316,31 @@ __device__ __forceinline__ int process_runs_t(const BuildParams& p, Shared& sh, 
         if (EVENTS) {
           add_event(dA, dB, sidx, c, 1u, P.combine);
           add_event(dA, dB, eidx, 0u - c, 0xffffffffu, P.combine);
+        }
+      }
+      if (dense) {
+        int key = seg;
+        u32 va = seg_all, vf = seg_full, vn = seg_cnt;
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+          const int kk = __shfl_up_sync(0xffffffffu, key, dd);
+          const u32 ya = __shfl_up_sync(0xffffffffu, va, dd), yf = __shfl_up_sync(0xffffffffu, vf, dd);
+          const u32 yn = __shfl_up_sync(0xffffffffu, vn, dd);
+          if (static_cast<int>(lane_id()) >= dd && kk == key) { va += ya; vf += yf; vn += yn; }
+        }
+        const int next_key = __shfl_down_sync(0xffffffffu, key, 1);
+        if (key != 0x7fffffff && (lane_id() == 31 || next_key != key)) {   // last lane of its round
+          const int si = buf * TILE + slot(key);
+          atomicAdd(&dA[si], va);
+          atomicAdd(&dB[si], vn & 0xffffu);
+          const u32 n_full = vn >> 16;
+          if (n_full && static_cast<off_t>(key) + trel + static_cast<off_t>(tau) < len) {
+            const u32 erel = static_cast<u32>(key) + tau;      // tau < TILE in dense phases
+            const int ei = erel < TILE ? buf * TILE + slot(static_cast<int>(erel))
+                                       : (buf ^ 1) * TILE + slot(static_cast<int>(erel - TILE));
+            atomicAdd(&dA[ei], 0u - vf);
+            atomicAdd(&dB[ei], 0u - n_full);
+          }
         }
       }
       acc.steps += steps;
@@ -458,14 +503,22 @@ __device__ __forceinline__ void write_jobs(const BuildParams& p, const Shared& s
       fin = oj <= sh.tau[0];
     }
     i64 start = -1, done = -1;
-    if (fin) {
+    {
       const i64 rank = may_carry ? static_cast<i64>(ec.fin_rank[pos]) : static_cast<i64>(pos - seg_lo - sh.ent[ph]);
       const i64 tau = sh.tau[ph], k = sh.k[ph];
-      start = sh.pbase[ph] + (simultaneous ? (rank / k) * tau : slot_offset(rank, tau, k));
-      done = start + oj;
-      acc.flow += done - (ec.ARR ? __ldg(ec.ARR + j) : 0);
-    } else {
-      ++acc.unfinished;
+      const i64 st = sh.pbase[ph] + (simultaneous ? (rank / k) * tau : slot_offset(rank, tau, k));
+      if (!may_carry) {   // exactly one run per job: its length and end are accounted here, not in the visit
+        const i64 d = fin ? oj : tau;
+        acc.steps += d;
+        acc.hmax = max_i64(acc.hmax, st + d);
+      }
+      if (fin) {
+        start = st;
+        done = st + oj;
+        acc.flow += done - (ec.ARR ? __ldg(ec.ARR + j) : 0);
+      } else {
+        ++acc.unfinished;
+      }
     }
     if (p.out.job_start) p.out.job_start[ec.job_out + j] = static_cast<int32_t>(start);
     if (p.out.job_completion) p.out.job_completion[ec.job_out + j] = static_cast<int32_t>(done);
@@ -596,6 +649,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
         // shared-memory atomics it saves unless a whole warp hits one word: only whole simultaneous
         // batches do that.
         P.combine = simultaneous && P.k >= 32;
+        P.dense = !simultaneous && P.tau < TILE && P.k >= 4 * P.tau;
         {
           u64 a_, b_;
           divmod_u(static_cast<u64>(P.tau), static_cast<u64>(P.k), &a_, &b_);
@@ -615,7 +669,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams 
 
         int C_next = 0;
         if (!P.profile_on) {
-          C_next = process_runs<false>(p, sh, ec, P, cur, nxt, 0, 0, N, 0, 0, acc);
+          if (P.may_carry || ec.want_runs)   // otherwise write_jobs does everything a run needs
+            C_next = process_runs<false>(p, sh, ec, P, cur, nxt, 0, 0, N, 0, 0, acc);
           if (event_form) {
             const i64* const ps = p.prefix_s + lo + st.instance + seg_lo;
             const i64 per = (static_cast<i64>(N) + T - 1) / T;
