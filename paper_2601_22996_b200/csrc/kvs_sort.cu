@@ -21,9 +21,16 @@ __device__ __forceinline__ int32_t key_at(const SortParams& p, i64 lo, int idx) 
   return p.key ? p.key[lo + idx] : p.o[lo + idx];
 }
 
+constexpr u32 COUNT_TAG = 0x80000000u;
+
+// Lanes of the warp holding the same value (a digit, or 256 for lanes past the end).
+__device__ __forceinline__ u32 match_digit(u32 digit) { return __match_any_sync(0xffffffffu, digit); }
+
 // Sort positions [seg_lo, seg_hi) of the instance starting at global job index lo.
+// cnt[digit][warp] (rows padded to 33 words: leaders of different digits and the column scans both
+// hit distinct banks) must hold no tagged entry on entry; it holds none on return.
 __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
-                             u32 (*warp_cnt)[256], u32* bucket, u32 (*hist)[256]) {
+                             u32 (*cnt)[WARPS + 1], u32* bucket, u32 (*hist)[256]) {
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n = seg_hi - seg_lo;
   int32_t* const out = p.perm + lo + seg_lo;
@@ -32,12 +39,17 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
     __syncthreads();
     return;
   }
-  // digit histograms of all passes in one sweep
+  // digit histograms of all passes in one sweep; lanes with equal digits add once per warp
   for (int i = tid; i < 4 * 256; i += T) (&hist[0][0])[i] = 0;
   __syncthreads();
-  for (int j = tid; j < n; j += T) {
-    u32 key = static_cast<u32>(key_at(p, lo, seg_lo + j));
-    for (int d = 0; d < passes; ++d) atomicAdd(&hist[d][(key >> (8 * d)) & 255u], 1u);
+  for (int j0 = 0; j0 < n; j0 += T) {
+    const int j = j0 + tid;
+    const u32 key = j < n ? static_cast<u32>(key_at(p, lo, seg_lo + j)) : 0u;
+    for (int d = 0; d < passes; ++d) {
+      const u32 digit = j < n ? (key >> (8 * d)) & 255u : 256u;
+      const u32 peers = match_digit(digit);
+      if (j < n && (peers & lanemask_lt()) == 0) atomicAdd(&hist[d][digit], static_cast<u32>(__popc(peers)));
+    }
   }
   __syncthreads();
   // exclusive scan of each histogram: warp d scans histogram d, 8 digits per lane
@@ -60,9 +72,8 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
     int32_t* dst = (to_perm ? p.perm : p.perm_tmp) + lo + seg_lo;
     const int32_t* src = (to_perm ? p.perm_tmp : p.perm) + lo + seg_lo;
     if (tid < 256) bucket[tid] = hist[pass][tid];
+    __syncthreads();
     for (int j0 = 0; j0 < n; j0 += T) {
-      for (int i = tid; i < WARPS * 256; i += T) (&warp_cnt[0][0])[i] = 0;
-      __syncthreads();
       const int j = j0 + tid;
       const bool valid = j < n;
       int idx = 0;
@@ -71,34 +82,47 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
         idx = pass == 0 ? seg_lo + j : src[j];
         digit = (static_cast<u32>(key_at(p, lo, idx)) >> (8 * pass)) & 255u;
       }
-      const u32 peers = __match_any_sync(0xffffffffu, digit);
+      const u32 peers = match_digit(digit);
       const u32 rank = __popc(peers & lanemask_lt());
-      if (valid && rank == 0) warp_cnt[warp][digit] = __popc(peers);
+      // count of this digit in this warp; the tag marks entries written for this tile (everything
+      // else in the table is an offset left by the previous tile's scan, tag clear)
+      if (valid && rank == 0) cnt[digit][warp] = static_cast<u32>(__popc(peers)) | COUNT_TAG;
       __syncthreads();
-      if (tid < 256) {
-        u32 acc = bucket[tid];
-        for (int w = 0; w < WARPS; ++w) {
-          u32 t = warp_cnt[w][tid];
-          warp_cnt[w][tid] = acc;
-          acc += t;
+      // column scans: warp w turns the 32 per-warp counts of digits 8w .. 8w+7 into positions
+      // behind the running bucket position, one lane per source warp
+#pragma unroll
+      for (int i = 0; i < 256 / WARPS; ++i) {
+        const int dg = warp * (256 / WARPS) + i;
+        const u32 raw = cnt[dg][lane_id()];
+        const u32 v = (raw & COUNT_TAG) ? (raw & ~COUNT_TAG) : 0u;
+        u32 incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const u32 y = __shfl_up_sync(0xffffffffu, incl, d);
+          if (static_cast<int>(lane_id()) >= d) incl += y;
         }
-        bucket[tid] = acc;
+        const u32 base = bucket[dg];
+        cnt[dg][lane_id()] = base + incl - v;
+        __syncwarp();
+        if (lane_id() == 31) bucket[dg] = base + incl;
       }
       __syncthreads();
-      if (valid) dst[warp_cnt[warp][digit] + rank] = idx;
+      if (valid) dst[cnt[digit][warp] + rank] = idx;
       __syncthreads();
     }
   }
 }
 
 __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
-  __shared__ u32 warp_cnt[WARPS][256];
+  __shared__ u32 cnt[256][WARPS + 1];
   __shared__ u32 hist[4][256];
   __shared__ u32 bucket[256];
   __shared__ int red[32];
   __shared__ i64 wsum[32];
   __shared__ int seg_end;
   const int tid = threadIdx.x;
+  for (int i = tid; i < 256 * (WARPS + 1); i += T) (&cnt[0][0])[i] = 0;
+  __syncthreads();
 
   for (i64 inst = blockIdx.x; inst < p.n_instances; inst += gridDim.x) {
     const i64 lo = p.job_off[inst], hi = p.job_off[inst + 1];
@@ -138,7 +162,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       }
       __syncthreads();
       const int seg_hi = seg_end;
-      sort_segment(p, lo, seg_lo, seg_hi, passes, warp_cnt, bucket, hist);
+      sort_segment(p, lo, seg_lo, seg_hi, passes, cnt, bucket, hist);
       __syncthreads();
       for (int j = seg_lo + tid; j < seg_hi; j += T) {
         const int idx = p.perm[lo + j];
