@@ -33,7 +33,8 @@ constexpr int TILE = KVS_TILE;
 constexpr int WARPS = T / 32;
 constexpr int RPT = 4;                     // consecutive ranks per thread in the run loop
 constexpr int CHUNK = T * RPT;
-static_assert(ITEMS == 8, "tile layout assumes two 4-word vectors per thread");
+constexpr int VEC = ITEMS / 4;              // 16-byte vectors per thread and tile
+static_assert(ITEMS % 4 == 0 && (ITEMS & (ITEMS - 1)) == 0, "rounds per thread: a power of two, whole vectors");
 
 typedef unsigned __int128 u128;
 
@@ -52,9 +53,10 @@ __device__ i64 max_parallelism(i64 tau, i64 s, i64 M) {
   return (k1 * D <= 2 * M - tau + gcd_i64(tau, k1)) ? k1 : k0;
 }
 
-// Shared-memory word of round e of a tile.  Thread t owns rounds 8t .. 8t+7 as two 4-word vectors;
-// vector c of thread t sits at vector index c*T + t, so a warp's vector access is contiguous.
-__device__ __forceinline__ int slot(int e) { return ((((e >> 2) & 1) * T + (e >> 3)) << 2) + (e & 3); }
+// Shared-memory word of round e of a tile.  Thread t owns rounds ITEMS*t .. ITEMS*t + ITEMS-1 as VEC
+// 4-word vectors; vector c of thread t sits at vector index c*T + t, so a warp's vector access is
+// contiguous.
+__device__ __forceinline__ int slot(int e) { return ((((e >> 2) % VEC) * T + e / ITEMS) << 2) + (e & 3); }
 
 struct Shared {
   uint4 dA[2][TILE / 4];    // two-tile ring: difference arrays of the constant terms
@@ -389,12 +391,15 @@ __device__ __forceinline__ void scan_tile(Shared& sh, int buf, i64 t0, int wlen,
                                           u32& A_run, u32& B_run, Acc& acc, const EvalCtx& ec, int32_t* profile) {
   const int tid = threadIdx.x;
   const uint4 zero = make_uint4(0, 0, 0, 0);
-  const uint4 a0 = sh.dA[buf][tid], a1 = sh.dA[buf][T + tid];
-  const uint4 b0 = sh.dB[buf][tid], b1 = sh.dB[buf][T + tid];
-  sh.dA[buf][tid] = zero; sh.dA[buf][T + tid] = zero;
-  sh.dB[buf][tid] = zero; sh.dB[buf][T + tid] = zero;
-  u32 a[ITEMS] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-  u32 b[ITEMS] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+  u32 a[ITEMS], b[ITEMS];
+#pragma unroll
+  for (int v = 0; v < VEC; ++v) {
+    const uint4 x = sh.dA[buf][v * T + tid], y = sh.dB[buf][v * T + tid];
+    sh.dA[buf][v * T + tid] = zero;
+    sh.dB[buf][v * T + tid] = zero;
+    a[4 * v] = x.x; a[4 * v + 1] = x.y; a[4 * v + 2] = x.z; a[4 * v + 3] = x.w;
+    b[4 * v] = y.x; b[4 * v + 1] = y.y; b[4 * v + 2] = y.z; b[4 * v + 3] = y.w;
+  }
 #pragma unroll
   for (int i = 1; i < ITEMS; ++i) { a[i] += a[i - 1]; b[i] += b[i - 1]; }
   const u32 sa = a[ITEMS - 1], sb = b[ITEMS - 1];
@@ -429,7 +434,7 @@ __device__ __forceinline__ void scan_tile(Shared& sh, int buf, i64 t0, int wlen,
     // rounds [lo, hi) of this tile belong to the phase and fit the caller's capacity
     const i64 lo = first_round, hi = min_i64(t0 + wlen, ec.prof_cap);
 #pragma unroll
-    for (int v = 0; v < 2; ++v) {
+    for (int v = 0; v < VEC; ++v) {
       const i64 rs = t0 + e0 + 4 * v;
       int32_t* dst = profile + ec.prof_base + rs;
       if (rs >= lo && rs + 4 <= hi) {
@@ -527,7 +532,7 @@ __device__ __forceinline__ void write_jobs(const BuildParams& p, const Shared& s
   }
 }
 
-__global__ void __launch_bounds__(KVS_EVAL_THREADS, 2) k_build_eval(BuildParams p) {
+__global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_eval(BuildParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   const int tid = threadIdx.x;

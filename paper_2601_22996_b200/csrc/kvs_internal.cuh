@@ -13,8 +13,14 @@ typedef unsigned int u32;
 
 constexpr int KVS_MAX_PHASES = 96;      // slices of one geometric ladder
 constexpr int KVS_SORT_THREADS = 1024;  // one CTA sorts one (instance, window) segment at a time
-constexpr int KVS_EVAL_THREADS = 512;   // one CTA per evaluation
-constexpr int KVS_EVAL_ITEMS = 8;       // rounds per thread and tile
+#ifndef KVS_EVAL_THREADS_CFG
+#define KVS_EVAL_THREADS_CFG 512
+#define KVS_EVAL_ITEMS_CFG 8
+#define KVS_EVAL_MIN_CTAS_CFG 2
+#endif
+constexpr int KVS_EVAL_THREADS = KVS_EVAL_THREADS_CFG;    // one CTA per evaluation
+constexpr int KVS_EVAL_ITEMS = KVS_EVAL_ITEMS_CFG;        // rounds per thread and tile
+constexpr int KVS_EVAL_MIN_CTAS = KVS_EVAL_MIN_CTAS_CFG;  // CTAs per SM the register allocation aims at
 constexpr int KVS_TILE = KVS_EVAL_THREADS * KVS_EVAL_ITEMS;  // rounds per shared-memory tile
 
 // Per-instance statistics produced by the first kernel.
