@@ -40,7 +40,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // one stream, so the entry points reuse the workspace from offset 0; the layout without staging
 // is a prefix of the layout with staging.
 struct Layout {
-  size_t settings, stats, perm, rec_a, rec_b, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter;
+  size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter;
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -53,8 +53,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.settings = take(static_cast<size_t>(P) * sizeof(kvs_setting));
   L.stats = take(static_cast<size_t>(I) * sizeof(InstStats));
   L.perm = take(static_cast<size_t>(N) * 4);
-  L.rec_a = take(static_cast<size_t>(N) * 8);
-  L.rec_b = take(static_cast<size_t>(N) * 8);
+  L.perm_tmp = take(static_cast<size_t>(N) * 4);
   L.sorted_s = take(static_cast<size_t>(N) * 4);
   L.sorted_o = take(static_cast<size_t>(N) * 4);
   L.sorted_key = take(static_cast<size_t>(N) * 4);
@@ -90,7 +89,7 @@ size_t generic_bytes(int64_t cap_total, int64_t P, size_t* second) {
 }
 
 struct SweepLayout {
-  size_t stats, perm, rec_a, rec_b, sorted_s, sorted_o, prefix_s, prefix_o, tau, k, acc_peak, acc_flow, total;
+  size_t stats, perm, perm_tmp, sorted_s, sorted_o, prefix_s, prefix_o, tau, k, acc_peak, acc_flow, total;
 };
 
 SweepLayout make_sweep_layout(int64_t N, int64_t max_n) {
@@ -99,8 +98,7 @@ SweepLayout make_sweep_layout(int64_t N, int64_t max_n) {
   auto take = [&](size_t bytes) { size_t r = at; at += align_up(bytes); return r; };
   L.stats = take(sizeof(InstStats));
   L.perm = take(static_cast<size_t>(N) * 4);
-  L.rec_a = take(static_cast<size_t>(N) * 8);
-  L.rec_b = take(static_cast<size_t>(N) * 8);
+  L.perm_tmp = take(static_cast<size_t>(N) * 4);
   L.sorted_s = take(static_cast<size_t>(N) * 4);
   L.sorted_o = take(static_cast<size_t>(N) * 4);
   L.prefix_s = take(static_cast<size_t>(max_n + 1) * 8);
@@ -196,8 +194,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   sp.window = inst->window; sp.n_instances = I; sp.max_jobs = max_n; sp.need_order = need_order ? 1 : 0;
   sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
   sp.perm = reinterpret_cast<int32_t*>(ws + L.perm);
-  sp.rec_a = reinterpret_cast<u64*>(ws + L.rec_a);
-  sp.rec_b = reinterpret_cast<u64*>(ws + L.rec_b);
+  sp.perm_tmp = reinterpret_cast<int32_t*>(ws + L.perm_tmp);
   sp.iperm = reinterpret_cast<int32_t*>(ws + L.iperm);
   sp.sorted_s = reinterpret_cast<int32_t*>(ws + L.sorted_s);
   sp.sorted_o = reinterpret_cast<int32_t*>(ws + L.sorted_o);
@@ -437,8 +434,7 @@ int kvs_sweep(kvs_ctx* ctx, const kvs_instances* inst, const kvs_sweep_params* p
   sp.window = 0; sp.n_instances = 1; sp.max_jobs = max_n; sp.need_order = 1;
   sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
   sp.perm = reinterpret_cast<int32_t*>(ws + L.perm);
-  sp.rec_a = reinterpret_cast<u64*>(ws + L.rec_a);
-  sp.rec_b = reinterpret_cast<u64*>(ws + L.rec_b);
+  sp.perm_tmp = reinterpret_cast<int32_t*>(ws + L.perm_tmp);
   sp.sorted_s = reinterpret_cast<int32_t*>(ws + L.sorted_s);
   sp.sorted_o = reinterpret_cast<int32_t*>(ws + L.sorted_o);
   sp.sorted_key = nullptr;

@@ -74,8 +74,7 @@ struct SortParams {
   int need_order;           // 0: statistics only
   InstStats* stats;
   int32_t* perm;
-  u64* rec_a;               // two buffers of (key << 32 | job index) records, [n_jobs_total] each
-  u64* rec_b;
+  int32_t* perm_tmp;
   int32_t* iperm;           // inverse of perm (job index -> position), or NULL
   int32_t* sorted_s;
   int32_t* sorted_o;

@@ -8,8 +8,8 @@
 //
 // Each pass ranks one tile of 1024 jobs at a time: lanes with equal digits find each other with
 // a warp match, per-warp digit counts go to shared memory, one column scan per digit turns them
-// into offsets behind the running bucket position.  What moves is an 8-byte record (key, job
-// index), so the passes read contiguously and the keys are gathered only once.
+// into offsets behind the running bucket position.  Keys are re-read through the permutation
+// (they stay in L2 for instances of this size), so only 4 bytes per job move per pass.
 #include "kvs_internal.cuh"
 
 namespace {
@@ -21,36 +21,23 @@ __device__ __forceinline__ int32_t key_at(const SortParams& p, i64 lo, int idx) 
   return p.key ? p.key[lo + idx] : p.o[lo + idx];
 }
 
-constexpr u32 COUNT_TAG = 0x80000000u;
-
-// Lanes of the warp holding the same value (a digit, or 256 for lanes past the end).
-__device__ __forceinline__ u32 match_digit(u32 digit) { return __match_any_sync(0xffffffffu, digit); }
-
 // Sort positions [seg_lo, seg_hi) of the instance starting at global job index lo.
-// cnt[digit][warp] (rows padded to 33 words: leaders of different digits and the column scans both
-// hit distinct banks) must hold no tagged entry on entry; it holds none on return.
-__device__ const u64* sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
-                             u32 (*cnt)[WARPS + 1], u32* bucket, u32 (*hist)[256]) {
+__device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
+                             u32 (*warp_cnt)[256], u32* bucket, u32 (*hist)[256]) {
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n = seg_hi - seg_lo;
+  int32_t* const out = p.perm + lo + seg_lo;
   if (passes == 0 || n <= 1) {
-    u64* const out = p.rec_a + lo + seg_lo;
-    for (int j = tid; j < n; j += T)
-      out[j] = (static_cast<u64>(static_cast<u32>(key_at(p, lo, seg_lo + j))) << 32) | static_cast<u32>(seg_lo + j);
+    for (int j = tid; j < n; j += T) out[j] = seg_lo + j;
     __syncthreads();
-    return out;
+    return;
   }
-  // digit histograms of all passes in one sweep; lanes with equal digits add once per warp
+  // digit histograms of all passes in one sweep
   for (int i = tid; i < 4 * 256; i += T) (&hist[0][0])[i] = 0;
   __syncthreads();
-  for (int j0 = 0; j0 < n; j0 += T) {
-    const int j = j0 + tid;
-    const u32 key = j < n ? static_cast<u32>(key_at(p, lo, seg_lo + j)) : 0u;
-    for (int d = 0; d < passes; ++d) {
-      const u32 digit = j < n ? (key >> (8 * d)) & 255u : 256u;
-      const u32 peers = match_digit(digit);
-      if (j < n && (peers & lanemask_lt()) == 0) atomicAdd(&hist[d][digit], static_cast<u32>(__popc(peers)));
-    }
+  for (int j = tid; j < n; j += T) {
+    u32 key = static_cast<u32>(key_at(p, lo, seg_lo + j));
+    for (int d = 0; d < passes; ++d) atomicAdd(&hist[d][(key >> (8 * d)) & 255u], 1u);
   }
   __syncthreads();
   // exclusive scan of each histogram: warp d scans histogram d, 8 digits per lane
@@ -67,68 +54,51 @@ __device__ const u64* sort_segment(const SortParams& p, i64 lo, int seg_lo, int 
   }
   __syncthreads();
 
-  // Records (key << 32 | job index) move between two buffers, so every pass reads contiguously and
-  // never goes back to the keys; the record of the next tile is requested before this tile is
-  // ranked, which hides the load latency behind the three barriers of a tile.
   for (int pass = 0; pass < passes; ++pass) {
-    u64* dst = ((pass & 1) ? p.rec_b : p.rec_a) + lo + seg_lo;
-    const u64* src = ((pass & 1) ? p.rec_a : p.rec_b) + lo + seg_lo;
+    // the last pass must land in perm: passes alternate between the two buffers
+    const bool to_perm = ((passes - 1 - pass) & 1) == 0;
+    int32_t* dst = (to_perm ? p.perm : p.perm_tmp) + lo + seg_lo;
+    const int32_t* src = (to_perm ? p.perm_tmp : p.perm) + lo + seg_lo;
     if (tid < 256) bucket[tid] = hist[pass][tid];
-    __syncthreads();
-    auto fetch = [&](int j) -> u64 {
-      if (j >= n) return 0;
-      if (pass > 0) return src[j];
-      return (static_cast<u64>(static_cast<u32>(key_at(p, lo, seg_lo + j))) << 32) | static_cast<u32>(seg_lo + j);
-    };
-    u64 rec_next = fetch(tid);
     for (int j0 = 0; j0 < n; j0 += T) {
+      for (int i = tid; i < WARPS * 256; i += T) (&warp_cnt[0][0])[i] = 0;
+      __syncthreads();
       const int j = j0 + tid;
       const bool valid = j < n;
-      const u64 idx = rec_next;           // the whole record travels
-      rec_next = fetch(j + T);
-      const u32 digit = valid ? static_cast<u32>(idx >> (32 + 8 * pass)) & 255u : 256u;   // 256: lanes past the end
-      const u32 peers = match_digit(digit);
+      int idx = 0;
+      u32 digit = 256;  // sentinel for lanes past the end
+      if (valid) {
+        idx = pass == 0 ? seg_lo + j : src[j];
+        digit = (static_cast<u32>(key_at(p, lo, idx)) >> (8 * pass)) & 255u;
+      }
+      const u32 peers = __match_any_sync(0xffffffffu, digit);
       const u32 rank = __popc(peers & lanemask_lt());
-      // count of this digit in this warp; the tag marks entries written for this tile (everything
-      // else in the table is an offset left by the previous tile's scan, tag clear)
-      if (valid && rank == 0) cnt[digit][warp] = static_cast<u32>(__popc(peers)) | COUNT_TAG;
+      if (valid && rank == 0) warp_cnt[warp][digit] = __popc(peers);
       __syncthreads();
-      // column scans: warp w turns the 32 per-warp counts of digits 8w .. 8w+7 into positions
-      // behind the running bucket position, one lane per source warp
-#pragma unroll
-      for (int i = 0; i < 256 / WARPS; ++i) {
-        const int dg = warp * (256 / WARPS) + i;
-        const u32 raw = cnt[dg][lane_id()];
-        const u32 v = (raw & COUNT_TAG) ? (raw & ~COUNT_TAG) : 0u;
-        u32 incl = v;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          const u32 y = __shfl_up_sync(0xffffffffu, incl, d);
-          if (static_cast<int>(lane_id()) >= d) incl += y;
+      if (tid < 256) {
+        u32 acc = bucket[tid];
+        for (int w = 0; w < WARPS; ++w) {
+          u32 t = warp_cnt[w][tid];
+          warp_cnt[w][tid] = acc;
+          acc += t;
         }
-        const u32 base = bucket[dg];
-        cnt[dg][lane_id()] = base + incl - v;
-        __syncwarp();
-        if (lane_id() == 31) bucket[dg] = base + incl;
+        bucket[tid] = acc;
       }
       __syncthreads();
-      if (valid) dst[cnt[digit][warp] + rank] = idx;
+      if (valid) dst[warp_cnt[warp][digit] + rank] = idx;
       __syncthreads();
     }
   }
-  return (((passes - 1) & 1) ? p.rec_b : p.rec_a) + lo + seg_lo;
 }
 
 __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
-  __shared__ u32 cnt[256][WARPS + 1];
+  __shared__ u32 warp_cnt[WARPS][256];
   __shared__ u32 hist[4][256];
   __shared__ u32 bucket[256];
   __shared__ int red[32];
   __shared__ i64 wsum[32];
   __shared__ int seg_end;
   const int tid = threadIdx.x;
-  for (int i = tid; i < 256 * (WARPS + 1); i += T) (&cnt[0][0])[i] = 0;
-  __syncthreads();
 
   for (i64 inst = blockIdx.x; inst < p.n_instances; inst += gridDim.x) {
     const i64 lo = p.job_off[inst], hi = p.job_off[inst + 1];
@@ -168,16 +138,13 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       }
       __syncthreads();
       const int seg_hi = seg_end;
-      const u64* const sorted = sort_segment(p, lo, seg_lo, seg_hi, passes, cnt, bucket, hist);
+      sort_segment(p, lo, seg_lo, seg_hi, passes, warp_cnt, bucket, hist);
       __syncthreads();
       for (int j = seg_lo + tid; j < seg_hi; j += T) {
-        const u64 rec = sorted[j - seg_lo];
-        const int idx = static_cast<int>(static_cast<u32>(rec));
-        const int key = static_cast<int>(rec >> 32);
-        p.perm[lo + j] = idx;
+        const int idx = p.perm[lo + j];
         p.sorted_s[lo + j] = p.s[lo + idx];
-        p.sorted_o[lo + j] = p.key ? p.o[lo + idx] : key;
-        if (p.key) p.sorted_key[lo + j] = key;
+        p.sorted_o[lo + j] = p.o[lo + idx];
+        if (p.key) p.sorted_key[lo + j] = p.key[lo + idx];
         if (p.iperm) p.iperm[lo + idx] = j;
       }
       __syncthreads();
