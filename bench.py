@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5", choices=sorted(WORKLOADS))
     ap.add_argument("--instances", type=int, default=0, help="override the number of instances (0 = the config's)")
+    ap.add_argument("--families", default="", help="comma-separated subset of the workload's families (diagnostic)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -64,9 +65,9 @@ def make_instances(name: str, n_inst: int, device, first_instance: int = 0):
     return workloads.Instances(off, cat("s"), cat("o"), cat("o_est"), cat("arrival"), meta)
 
 
-def make_settings(name: str, inst):
+def make_settings(name: str, inst, fams=None):
     from paper_2601_22996_b200 import binding
-    fams = WORKLOADS[name][3]
+    fams = fams or WORKLOADS[name][3]
     I = inst.n_instances
     if "M_per_instance" in inst.meta:
         Ms = inst.meta["M_per_instance"].cpu().numpy()[:, None]
@@ -184,11 +185,11 @@ def run_ours(args):
     name = args.workload
     I = args.instances or WORKLOADS[name][1]
     n = WORKLOADS[name][2]
-    fams = WORKLOADS[name][3]
+    fams = [f for f in args.families.split(",") if f] or WORKLOADS[name][3]
 
     # weak scaling: every rank gets its own I instances (different seeds), no data-path collective
     inst = make_instances(name, I, dev, first_instance=rank * I)
-    settings, window = make_settings(name, inst)
+    settings, window = make_settings(name, inst, fams)
     P = settings.shape[0]
     N = I * n
     sched = Scheduler(local)

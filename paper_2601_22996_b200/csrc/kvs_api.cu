@@ -14,6 +14,7 @@ struct kvs_ctx {
   uint64_t workspace_bytes = 0;
   int sm_count = 0;
   int build_ctas_per_sm = 1;
+  int fused_ctas_per_sm = 1;
   bool timing = false;
   bool timed = false;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before the ordering kernel, between, after the builder
@@ -40,7 +41,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // one stream, so the entry points reuse the workspace from offset 0; the layout without staging
 // is a prefix of the layout with staging.
 struct Layout {
-  size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter;
+  size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter, slow_list;
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -60,9 +61,10 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.prefix_s = take(static_cast<size_t>(N + I) * 8);
   L.iperm = take(static_cast<size_t>(N) * 4);
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
-  L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 4);
+  L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 8);   // (s, o) pairs in the fast kernel
   L.fin_rank = take(static_cast<size_t>(grid) * static_cast<size_t>(max_n) * 4);
-  L.counter = take(8);
+  L.counter = take(32);   // work counter of the fast kernel, length of its left-over list, work counter of the general kernel
+  L.slow_list = take(static_cast<size_t>(P) * 8);
   if (staging) {
     L.st_off = take(static_cast<size_t>(I + 1) * 8);
     L.st_s = take(static_cast<size_t>(N) * 4);
@@ -223,11 +225,28 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.settings = reinterpret_cast<const kvs_setting*>(ws + L.settings);
   bp.P = P; bp.out = o; bp.ev = v; bp.do_profile = do_profile;
   bp.lists = reinterpret_cast<int32_t*>(ws + L.lists);
-  bp.counter = reinterpret_cast<ull*>(ws + L.counter);
-  int64_t grid = static_cast<int64_t>(ctx->sm_count) * ctx->build_ctas_per_sm;
-  if (grid > KVS_MAX_GRID) grid = KVS_MAX_GRID;
-  if (grid > P) grid = P;
-  ce = kvs_launch_build(bp, static_cast<int>(grid), ctx->stream);
+  ull* const counters = reinterpret_cast<ull*>(ws + L.counter);
+  auto grid_for = [&](int ctas_per_sm) {
+    int64_t g = static_cast<int64_t>(ctx->sm_count) * ctas_per_sm;
+    if (g > KVS_MAX_GRID) g = KVS_MAX_GRID;
+    if (g > P) g = P;
+    return static_cast<int>(g);
+  };
+  // The 32-bit fast kernel covers calls that want neither the explicit run list nor 64-bit job
+  // results; evaluations it cannot finish (times of 2^31 or more, memory bound of 2^32 or more)
+  // come back in a list that the general kernel works off.  Other calls go to the general kernel.
+  const bool fast = !run_out && !o.job_start64 && !o.job_completion64;
+  if (fast) {
+    bp.counter = counters;
+    bp.slow_count = counters + 1;
+    bp.slow_list = reinterpret_cast<i64*>(ws + L.slow_list);
+    ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), ctx->stream);
+    if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    bp.eval_list = bp.slow_list;
+    bp.eval_count = bp.slow_count;
+  }
+  bp.counter = counters + 2;
+  ce = kvs_launch_build(bp, grid_for(ctx->build_ctas_per_sm), ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "build launch");
   if (ctx->timing) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; }
   return KVS_OK;
@@ -258,6 +277,7 @@ int kvs_init(const kvs_init_params* params, kvs_ctx** out) {
   }
   ctx->sm_count = prop.multiProcessorCount;
   ctx->build_ctas_per_sm = kvs_build_ctas_per_sm();
+  ctx->fused_ctas_per_sm = kvs_fused_ctas_per_sm();
   *out = ctx;
   return KVS_OK;
 }

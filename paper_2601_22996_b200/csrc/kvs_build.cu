@@ -547,8 +547,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_e
     __syncthreads();  // previous evaluation done with shared memory
     if (tid == 0) sh.next_eval = static_cast<i64>(atomicAdd(reinterpret_cast<ull*>(p.counter), 1ull));
     __syncthreads();
-    const i64 e = sh.next_eval;
-    if (e >= p.P) break;
+    const i64 slot_no = sh.next_eval;
+    if (slot_no >= (p.eval_list ? static_cast<i64>(*p.eval_count) : p.P)) break;
+    const i64 e = p.eval_list ? p.eval_list[slot_no] : slot_no;
     const kvs_setting st = p.settings[e];
     const i64 lo = p.job_off[st.instance];
     const InstStats stats = p.stats[st.instance];

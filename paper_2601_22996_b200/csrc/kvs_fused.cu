@@ -1,0 +1,807 @@
+// Fused schedule builder and evaluator, 32-bit fast path: one CTA per (instance, setting, family)
+// evaluation, times below 2^31.
+//
+// For one evaluation (and one arrival window at a time) the CTA
+//   1. forms the phase table: the geometric ladder tau_p with the largest memory-feasible
+//      parallelism k_p (first line of the two geometric algorithms; Lemma "Peak Memory Usage of
+//      SPS"; Eq. max-parallelism), or the single (tau, k) of SPS / SimS;
+//   2. plans the phases without touching a run: a job enters at the class f of its key and leaves
+//      at the class l of the larger of key and response length, so phase p has
+//      N_p = #{f <= p} - #{l < p} participants; that fixes every phase's length
+//      floor((N_p - 1) tau_p / k_p) + tau_p and first round;
+//   3. writes every job's start and completion: the job's rank in the phase that completes it is
+//      the number of earlier positions (in schedule order) that leave in that phase or later; for
+//      exact keys that is the position inside the class, otherwise it is counted with one warp
+//      ballot per phase over 32 positions at a time, behind per-warp class histograms.
+//      start = base_p + floor(r*tau_p/k_p) (Procedure StaggeredPipelineSchedule) or
+//      base + floor(r/k)*tau (simultaneous batches), completion = start + o;
+//   4. if the memory profile is wanted, walks the phases tile by tile as the general kernel does:
+//      the runs that start inside a tile are a contiguous rank range, every run adds (c, 1) at its
+//      first round and (-c, -1) after its last one to two shared-memory difference arrays
+//      (c = s + 1 - start), one scan per array gives memory(t) = A(t) + t*B(t)
+//      (Eq. Memory-Feasibility), the peak is reduced and the profile stored 16 bytes at a time.
+//      Jobs killed at the end of their slot are carried to the next phase as (s, o) pairs, so a
+//      phase reads its participants as one contiguous stream.
+//
+// An evaluation whose times reach 2^31 or whose memory bound reaches 2^32 is not finished here: its
+// index is appended to a list that the general kernel works off afterwards.
+#include "kvs_events.cuh"
+
+namespace {
+
+constexpr int T = KVS_EVAL_THREADS;
+constexpr int ITEMS = KVS_EVAL_ITEMS;
+constexpr int TILE = KVS_TILE;
+constexpr int WARPS = T / 32;
+constexpr int VEC = ITEMS / 4;
+constexpr int RPT = 4;                       // consecutive ranks per thread in the run visit
+constexpr int MAXP = KVS_MAX_PHASES;
+constexpr u32 TIME_LIMIT = 0x7fffffffu - 4u * TILE;   // phase ends stay below this
+
+typedef unsigned __int128 u128;
+
+struct FShared {
+  uint4 dA[2][TILE / 4];      // two-tile ring: difference arrays of the constant terms
+  uint4 dB[2][TILE / 4];      //                and of the slopes
+  u128 pw_a[MAXP + 1];
+  u128 pw_b[MAXP + 1];
+  u64 taupre[MAXP + 1];       // sum of tau_q over q < p
+  i64 plen[MAXP];
+  i64 red64[32];
+  i64 next_eval;
+  i64 base_next;
+  i64 n_runs;
+  u32 tau[MAXP], k[MAXP], pbase[MAXP], np[MAXP];
+  u32 cnt[WARPS][MAXP];       // per-warp class counts, then ranks before each warp's segment
+  u32 redA[32], redB[32];
+  int red32[32];
+  int ent[MAXP + 1];          // class boundaries in key order
+  int n_phases, seg_end, fallback;
+};
+
+__device__ __forceinline__ u32 gcd_u32(u32 x, u32 y) {
+  while (y) { const u32 t = x % y; x = y; y = t; }
+  return x;
+}
+
+// Largest k >= 1 with s*k + (tau*k + tau + k - gcd(tau, k))/2 <= M, given s + tau <= M: the
+// condition reads k*(2s+tau+1) <= 2M - tau + gcd(tau,k), and 1 <= gcd <= tau leaves k0 or k0 + 1
+// with k0 = floor((2M - tau + 1) / (2s + tau + 1)).
+__device__ u32 max_parallelism32(u32 tau, u32 s, u32 M) {
+  const u64 D = 2ull * s + tau + 1ull;
+  const u64 num = 2ull * M - tau + 1ull;
+  u64 k0, r;
+  divmod_u(num, D, &k0, &r);
+  const u64 k1 = k0 + 1;
+  if (k1 >> 31) return static_cast<u32>(k0);
+  return (k1 * D <= 2ull * M - tau + gcd_u32(tau, static_cast<u32>(k1))) ? static_cast<u32>(k1) : static_cast<u32>(k0);
+}
+
+__device__ void ladder32(FShared& sh, i64 X, int a, int b, i64 beta0, u32 s_bar, u32 M) {
+  const int lane = lane_id();
+  if (beta0 <= 0) {
+    if (lane == 0) {
+      u128 pa = 1, pb = 1;
+      int ell = 0;
+      sh.pw_a[0] = 1; sh.pw_b[0] = 1;
+      while (ell + 1 < MAXP + 1) {
+        const u128 na = pa * static_cast<u128>(a), nb = pb * static_cast<u128>(b);
+        if (na > static_cast<u128>(X) * nb) break;
+        pa = na; pb = nb; ++ell;
+        sh.pw_a[ell] = pa; sh.pw_b[ell] = pb;
+      }
+      sh.n_phases = (ell + 1 <= MAXP) ? ell + 1 : 0;
+    }
+    __syncwarp();
+    const int L = sh.n_phases;
+    for (int p = lane; p < L; p += 32) {
+      const int j = L - 1 - p;  // tau_p = floor(X * b^j / a^j)
+      const u32 t = (a == 2 && b == 1) ? static_cast<u32>(X >> j)
+                                       : static_cast<u32>(static_cast<u128>(X) * sh.pw_b[j] / sh.pw_a[j]);
+      sh.tau[p] = t;
+      sh.k[p] = max_parallelism32(t, s_bar, M);
+    }
+  } else {
+    if (lane == 0) {
+      u128 pa = 1, pb = 1;
+      int p = 0;
+      for (;; ++p) {
+        if (p >= MAXP) { p = -1; break; }
+        const u128 num = static_cast<u128>(beta0) * pa;   // tau_p = min(floor(beta0 * a^p / b^p), X)
+        const u32 t = (num >= static_cast<u128>(X) * pb) ? static_cast<u32>(X) : static_cast<u32>(num / pb);
+        sh.tau[p] = t;
+        sh.k[p] = max_parallelism32(t, s_bar, M);
+        if (t >= X) break;
+        pa *= static_cast<u128>(a); pb *= static_cast<u128>(b);
+      }
+      sh.n_phases = p + 1;
+    }
+  }
+  __syncwarp();
+}
+
+// class(v) = first p with tau_p >= v (tau is nondecreasing and tau_(L-1) >= v)
+__device__ __forceinline__ int class_of(const u32* tau, int L, u32 v) {
+  int a = 0, b = L - 1;
+  while (a < b) { const int m = (a + b) >> 1; if (tau[m] >= v) b = m; else a = m + 1; }
+  return a;
+}
+
+// floor(r * tau / k) for r, tau, k below 2^31 with a result below 2^31
+__device__ __forceinline__ u32 slot32(u32 r, u32 tau, u32 k) {
+  const u64 x = static_cast<u64>(r) * tau;
+  if ((x >> 32) == 0) return static_cast<u32>(x) / k;
+  return static_cast<u32>(x / k);
+}
+
+// Word of round e of a tile: thread t owns rounds ITEMS*t .. ITEMS*t+ITEMS-1 as VEC 4-word vectors,
+// vector c of thread t at vector index c*T + t, so that a warp's vector access is contiguous.
+__device__ __forceinline__ int slot(int e) { return ((((e >> 2) % VEC) * T + e / ITEMS) << 2) + (e & 3); }
+// Word of the round `rel` rounds after the origin of ring half `buf`, 0 <= rel < 2*TILE.
+__device__ __forceinline__ int ring(int buf, int rel) { return ((buf ^ (rel >= TILE ? 1 : 0)) * TILE) + slot(rel & (TILE - 1)); }
+
+__device__ __forceinline__ int block_count_scan(int v, int* red32, int* total) {
+  int incl = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, d);
+    if (static_cast<int>(lane_id()) >= d) incl += y;
+  }
+  const int warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane_id() == 31) red32[warp] = incl;
+  __syncthreads();
+  const int w = (lane_id() < WARPS) ? red32[lane_id()] : 0;
+  int wi = w;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, wi, d);
+    if (static_cast<int>(lane_id()) >= d) wi += y;
+  }
+  *total = __shfl_sync(0xffffffffu, wi, 31);
+  return __shfl_sync(0xffffffffu, wi - w, warp) + (incl - v);
+}
+
+// One phase as the run visit sees it.  Participants in rank order: `C` carried (s, o) pairs in
+// `cur`, then the positions src_lo .. of the instance's schedule order.
+struct PhaseView {
+  const uint2* cur;
+  const int32_t* S;
+  const int32_t* O;
+  int C;
+  u32 tau, k, qt, rt;     // tau = qt*k + rt
+  u32 len;                // rounds of the phase
+  u32 base;               // its first round
+};
+
+// Visits ranks [ra, rb), all of which start inside the tile whose origin is `trel` rounds after
+// the phase's first round (trel may be slightly negative) and whose ring half is `buf`: adds the
+// two events of every run and appends the killed jobs to `nxt`.  Returns the new length of `nxt`.
+template <bool SIM, bool CARRY>
+__device__ __forceinline__ int visit_runs(FShared& sh, const PhaseView& P, uint2* nxt, int C_next,
+                                          int ra, int rb, int trel, int buf, bool dense, bool combine) {
+  const int tid = threadIdx.x;
+  u32* const dA = reinterpret_cast<u32*>(sh.dA);
+  u32* const dB = reinterpret_cast<u32*>(sh.dB);
+  const u32 tau = P.tau, k = P.k;
+  for (int c0 = ra; c0 < rb;) {
+    const int left = rb - c0;
+    const int rpt = left > 2 * T ? RPT : (left > T ? 2 : 1);
+    const int r_first = c0 + tid * rpt;
+    c0 += T * rpt;
+    uint2 keep[RPT];
+    u32 cmask = 0;
+    if (r_first - static_cast<int>(lane_id()) * rpt < rb) {   // warps past the end of the range skip the visit
+      u32 s_[RPT], o_[RPT];
+      bool on[RPT];
+#pragma unroll
+      for (int j = 0; j < RPT; ++j) {
+        const int r = r_first + j;
+        on[j] = j < rpt && r < rb;
+        s_[j] = 0; o_[j] = 0;
+        if (on[j]) {
+          if (r < P.C) { const uint2 e = P.cur[r]; s_[j] = e.x; o_[j] = e.y; }
+          else { s_[j] = static_cast<u32>(__ldg(P.S + (r - P.C))); o_[j] = static_cast<u32>(__ldg(P.O + (r - P.C))); }
+        }
+      }
+      u32 q = 0, rem = 0;      // start offset of the current rank inside the phase and its remainder
+      if (on[0]) {
+        if (SIM) {
+          const u32 b = static_cast<u32>(r_first) / k;
+          q = b * tau;
+          rem = static_cast<u32>(r_first) - b * k;
+        } else {
+          u64 dq_, dr_;
+          divmod_u(static_cast<u64>(r_first) * tau, k, &dq_, &dr_);
+          q = static_cast<u32>(dq_);
+          rem = static_cast<u32>(dr_);
+        }
+      }
+      // Dense phases (several runs start per round): the runs of a lane that start in the round of
+      // its first run are summed in registers, then equal rounds - contiguous lanes, because
+      // consecutive ranks start in nondecreasing rounds - are summed across the warp with a
+      // segmented scan, and one lane per round issues the atomics.  Runs that hold their whole
+      // slot end together (start + tau), so their end events are combined the same way.
+      const bool dn = !SIM && dense;
+      int seg = 0x7fffffff;
+      u32 seg_all = 0, seg_full = 0, seg_cnt = 0;
+#pragma unroll
+      for (int j = 0; j < RPT; ++j) {
+        int sidx = -1, eidx = -1;
+        u32 c = 0;
+        if (on[j]) {
+          const u32 oi = o_[j];
+          const u32 d = oi < tau ? oi : tau;
+          if (CARRY && oi > tau) { keep[j] = make_uint2(s_[j], oi); cmask |= 1u << j; }
+          c = s_[j] + 1u - P.base - q;                          // tokens(t) = c + t while active
+          const int srel = static_cast<int>(q) - trel;
+          sidx = ring(buf, srel);
+          if (q + d < P.len) {                                   // an end at the phase end is never read
+            const u32 erel = static_cast<u32>(srel) + d;
+            if (erel < 2u * TILE) eidx = ring(buf, static_cast<int>(erel));
+          }
+          if (dn) {
+            if (seg == 0x7fffffff) seg = srel;
+            if (srel == seg) {
+              seg_all += c; seg_cnt += 1u;
+              sidx = -1;
+              if (d == tau) { seg_full += c; seg_cnt += 1u << 16; eidx = -1; }
+            }
+          }
+          if (SIM) { if (++rem == k) { rem = 0; q += tau; } }
+          else { rem += P.rt; q += P.qt; if (rem >= k) { rem -= k; ++q; } }
+        }
+        if (SIM && combine) {
+          // whole simultaneous batches hit one word: sum equal targets inside the warp first
+          const u32 ps = __match_any_sync(0xffffffffu, sidx);
+          if (sidx >= 0) {
+            const u32 cs = __reduce_add_sync(ps, c);
+            if ((ps & lanemask_lt()) == 0) { atomicAdd(&dA[sidx], cs); atomicAdd(&dB[sidx], static_cast<u32>(__popc(ps))); }
+          }
+          const u32 pe = __match_any_sync(0xffffffffu, eidx);
+          if (eidx >= 0) {
+            const u32 ce = __reduce_add_sync(pe, c);
+            if ((pe & lanemask_lt()) == 0) { atomicAdd(&dA[eidx], 0u - ce); atomicAdd(&dB[eidx], 0u - static_cast<u32>(__popc(pe))); }
+          }
+        } else {
+          if (sidx >= 0) { atomicAdd(&dA[sidx], c); atomicAdd(&dB[sidx], 1u); }
+          if (eidx >= 0) { atomicAdd(&dA[eidx], 0u - c); atomicAdd(&dB[eidx], 0xffffffffu); }
+        }
+      }
+      if (dn) {
+        int key = seg;
+        u32 va = seg_all, vf = seg_full, vn = seg_cnt;
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+          const int kk = __shfl_up_sync(0xffffffffu, key, dd);
+          const u32 ya = __shfl_up_sync(0xffffffffu, va, dd), yf = __shfl_up_sync(0xffffffffu, vf, dd);
+          const u32 yn = __shfl_up_sync(0xffffffffu, vn, dd);
+          if (static_cast<int>(lane_id()) >= dd && kk == key) { va += ya; vf += yf; vn += yn; }
+        }
+        const int next_key = __shfl_down_sync(0xffffffffu, key, 1);
+        if (key != 0x7fffffff && (lane_id() == 31 || next_key != key)) {   // last lane of its round
+          const int si = ring(buf, key);
+          atomicAdd(&dA[si], va);
+          atomicAdd(&dB[si], vn & 0xffffu);
+          const u32 n_full = vn >> 16;
+          // start offset of this round inside the phase: key + trel
+          if (n_full && static_cast<u32>(key + trel) + tau < P.len) {
+            const int ei = ring(buf, key + static_cast<int>(tau));          // tau < TILE in dense phases
+            atomicAdd(&dA[ei], 0u - vf);
+            atomicAdd(&dB[ei], 0u - n_full);
+          }
+        }
+      }
+    }
+    if (CARRY) {
+      int total;
+      int off = C_next + block_count_scan(__popc(cmask), sh.red32, &total);
+#pragma unroll
+      for (int j = 0; j < RPT; ++j)
+        if (cmask >> j & 1u) nxt[off++] = keep[j];
+      C_next += total;
+    }
+  }
+  return C_next;
+}
+
+// Slices longer than a tile: ends that land two or more tiles after the run's start were not
+// inserted when the run was visited; pick them up when their tile comes.  u0 = offset of this
+// tile's origin inside the phase, a0 = the same for the phase's first tile (0 or slightly negative).
+__device__ __forceinline__ void insert_far_ends(FShared& sh, const PhaseView& P, bool sim, int N, int a0, int u0,
+                                                int wlen, int buf) {
+  if (u0 <= TILE) return;
+  const u32 lo = static_cast<u32>(u0) > P.tau ? static_cast<u32>(u0) - P.tau : 0u, hi = static_cast<u32>(u0 - TILE);
+  i64 r_lo, r_hi;   // ranks whose start offset lies in [lo, hi)
+  if (sim) { r_lo = ceil_div_u(lo, P.tau) * P.k; r_hi = ceil_div_u(hi, P.tau) * P.k; }
+  else { r_lo = ceil_div_u(static_cast<u64>(lo) * P.k, P.tau); r_hi = ceil_div_u(static_cast<u64>(hi) * P.k, P.tau); }
+  if (r_hi > N) r_hi = N;
+  u32* const dA = reinterpret_cast<u32*>(sh.dA);
+  u32* const dB = reinterpret_cast<u32*>(sh.dB);
+  for (i64 r0 = r_lo; r0 < r_hi; r0 += T) {
+    const i64 rr = r0 + threadIdx.x;
+    if (rr < r_hi) {
+      const int r = static_cast<int>(rr);
+      u32 si, oi;
+      if (r < P.C) { const uint2 e = P.cur[r]; si = e.x; oi = e.y; }
+      else { si = static_cast<u32>(__ldg(P.S + (r - P.C))); oi = static_cast<u32>(__ldg(P.O + (r - P.C))); }
+      const u32 q = sim ? (static_cast<u32>(r) / P.k) * P.tau : slot32(static_cast<u32>(r), P.tau, P.k);
+      const u32 end = q + (oi < P.tau ? oi : P.tau);
+      const int ts = a0 + ((static_cast<int>(q) - a0) / TILE) * TILE;   // origin of the tile the run started in
+      if (static_cast<int>(end) >= ts + 2 * TILE && static_cast<int>(end) >= u0 && static_cast<int>(end) < u0 + wlen && end < P.len) {
+        const u32 c = si + 1u - P.base - q;
+        const int ei = buf * TILE + slot(static_cast<int>(end) - u0);
+        atomicAdd(&dA[ei], 0u - c);
+        atomicAdd(&dB[ei], 0xffffffffu);
+      }
+    }
+  }
+}
+
+// Prefix-sums one tile of the ring, turns it into memory(t), reduces the peak, stores the profile
+// and leaves the tile zeroed for its next use.  Contains one __syncthreads.  t0 = absolute round
+// of the tile's origin; rounds [first_round, t0 + wlen) below prof_cap are stored.
+__device__ __forceinline__ void scan_tile(FShared& sh, int buf, i64 t0, int wlen, u32 first_round,
+                                          u32& A_run, u32& B_run, u32& peak, int32_t* prof, i64 prof_cap) {
+  const int tid = threadIdx.x;
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  u32 a[ITEMS], b[ITEMS];
+#pragma unroll
+  for (int v = 0; v < VEC; ++v) {
+    const uint4 x = sh.dA[buf][v * T + tid], y = sh.dB[buf][v * T + tid];
+    sh.dA[buf][v * T + tid] = zero;
+    sh.dB[buf][v * T + tid] = zero;
+    a[4 * v] = x.x; a[4 * v + 1] = x.y; a[4 * v + 2] = x.z; a[4 * v + 3] = x.w;
+    b[4 * v] = y.x; b[4 * v + 1] = y.y; b[4 * v + 2] = y.z; b[4 * v + 3] = y.w;
+  }
+#pragma unroll
+  for (int i = 1; i < ITEMS; ++i) { a[i] += a[i - 1]; b[i] += b[i - 1]; }
+  const u32 sa = a[ITEMS - 1], sb = b[ITEMS - 1];
+  u32 ia = sa, ib = sb;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 ya = __shfl_up_sync(0xffffffffu, ia, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
+    if (static_cast<int>(lane_id()) >= d) { ia += ya; ib += yb; }
+  }
+  if (lane_id() == 31) { sh.redA[tid >> 5] = ia; sh.redB[tid >> 5] = ib; }
+  __syncthreads();
+  const u32 wa = (lane_id() < WARPS) ? sh.redA[lane_id()] : 0, wb = (lane_id() < WARPS) ? sh.redB[lane_id()] : 0;
+  u32 wia = wa, wib = wb;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 ya = __shfl_up_sync(0xffffffffu, wia, d), yb = __shfl_up_sync(0xffffffffu, wib, d);
+    if (static_cast<int>(lane_id()) >= d) { wia += ya; wib += yb; }
+  }
+  const u32 offA = A_run + __shfl_sync(0xffffffffu, wia - wa, tid >> 5) + (ia - sa);
+  const u32 offB = B_run + __shfl_sync(0xffffffffu, wib - wb, tid >> 5) + (ib - sb);
+  A_run += __shfl_sync(0xffffffffu, wia, 31);
+  B_run += __shfl_sync(0xffffffffu, wib, 31);
+  const int e0 = tid * ITEMS;
+  const u32 tt = static_cast<u32>(t0) + static_cast<u32>(e0);
+  u32 mem[ITEMS];
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    mem[i] = (offA + a[i]) + (tt + i) * (offB + b[i]);
+    if (e0 + i < wlen) peak = max(peak, mem[i]);
+  }
+  if (prof_cap > 0) {
+    const i64 lo = first_round, hi = min_i64(t0 + wlen, prof_cap);
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) {
+      const i64 rs = t0 + e0 + 4 * v;
+      int32_t* dst = prof + rs;
+      if (rs >= lo && rs + 4 <= hi) {
+        *reinterpret_cast<int4*>(dst) = make_int4(static_cast<int>(mem[4 * v]), static_cast<int>(mem[4 * v + 1]),
+                                                  static_cast<int>(mem[4 * v + 2]), static_cast<int>(mem[4 * v + 3]));
+      } else if (rs + 4 > lo && rs < hi) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (rs + i >= lo && rs + i < hi) dst[i] = static_cast<int>(mem[4 * v + i]);
+      }
+    }
+  }
+}
+
+struct FAcc {
+  u64 flow = 0, steps = 0;
+  u32 hmax = 0;
+  int unfinished = 0;
+  u32 peak = 0;
+  i64 peak64 = 0;
+};
+
+__global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_eval(BuildParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  FShared& sh = *reinterpret_cast<FShared*>(smem_raw);
+  const int tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
+  uint2* const list0 = reinterpret_cast<uint2*>(p.lists) + static_cast<i64>(blockIdx.x) * 2 * p.max_jobs;
+  uint2* const list1 = list0 + p.max_jobs;
+  u32* const fin_start = reinterpret_cast<u32*>(p.fin_rank) + static_cast<i64>(blockIdx.x) * p.max_jobs;
+  {
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 2 * (TILE / 4); i += T) { (&sh.dA[0][0])[i] = zero; (&sh.dB[0][0])[i] = zero; }
+  }
+
+  for (;;) {
+    __syncthreads();
+    if (tid == 0) {
+      sh.next_eval = static_cast<i64>(atomicAdd(p.counter, 1ull));
+      sh.fallback = 0;
+      sh.n_runs = 0;
+    }
+    __syncthreads();
+    const i64 e = sh.next_eval;
+    if (e >= p.P) break;
+    const kvs_setting st = p.settings[e];
+    const i64 lo = p.job_off[st.instance];
+    const InstStats stats = p.stats[st.instance];
+    const int n = stats.flags ? 0 : static_cast<int>(p.job_off[st.instance + 1] - lo);
+    const i64 M = st.M;
+    const i64 s_bar = st.s_bar >= 0 ? st.s_bar : stats.s_max;
+    const i64 X = M - s_bar;
+    const int family = st.family;
+    const bool geometric = family == KVS_GBA || family == KVS_GSA;
+    const bool sim = family == KVS_SIMS;
+    const bool est = p.key != nullptr;
+    const bool keyed = !(family == KVS_GSA && !est);          // plain GSA keeps the index order
+    const bool carry = geometric && (family == KVS_GSA || est);
+    const bool est_class = est && family == KVS_GBA;          // classes by the clipped estimate
+    // arrays in schedule order (of the instance)
+    const int32_t* const S_ord = (keyed ? p.sorted_s : p.s) + lo;
+    const int32_t* const O_ord = (keyed ? p.sorted_o : p.o) + lo;
+    const int32_t* const K_ord = est ? p.sorted_key + lo : O_ord;
+    const int32_t* const IPERM = keyed ? p.iperm + lo : nullptr;
+    const int32_t* const O_JOB = p.o + lo;
+    const i64* const ARR = p.arrival ? p.arrival + lo : nullptr;
+    const i64 job_out = p.out.job_out_off ? p.out.job_out_off[e] : 0;
+    int32_t* const out_start = p.out.job_start ? p.out.job_start + job_out : nullptr;
+    int32_t* const out_done = p.out.job_completion ? p.out.job_completion + job_out : nullptr;
+    const i64 prof_base = p.ev.profile_off ? p.ev.profile_off[e] : 0;
+    const i64 prof_cap = (p.ev.profile && p.ev.profile_off) ? p.ev.profile_off[e + 1] - prof_base : 0;
+    int32_t* const prof = p.ev.profile ? p.ev.profile + prof_base : nullptr;
+    const bool want32 = p.out.job_start || p.out.job_completion;
+    const bool event_form = p.do_profile && !geometric && p.prefix_s != nullptr && prof_cap == 0;
+    const bool walk = p.do_profile && !event_form;            // rounds are walked tile by tile
+
+    int status = stats.flags;
+    if (!status && (X < 1 || stats.o_max > X)) status = KVS_EVAL_INFEASIBLE;
+    if (!status && geometric) {
+      if (tid < 32) ladder32(sh, X, st.alpha_num, st.alpha_den, st.beta0, static_cast<u32>(s_bar), static_cast<u32>(M));
+      __syncthreads();
+      if (sh.n_phases == 0) status = KVS_EVAL_RANGE;
+    }
+
+    FAcc acc;
+    i64 base = 0;          // first round of the next phase
+    i64 written_to = 0;    // profile rounds [0, written_to) have been written
+    bool give_up = false;
+
+    int seg_lo = 0;
+    while (!status && !give_up && seg_lo < n) {
+      // ---- window = offline sub-instance [seg_lo, seg_hi) ----
+      if (tid == 0) {
+        int end = n;
+        if (p.window > 0 && ARR) {
+          const i64 limit = (ARR[seg_lo] / p.window + 1) * p.window;
+          int a = seg_lo + 1, b = n;
+          while (a < b) { const int m = (a + b) >> 1; if (ARR[m] < limit) a = m + 1; else b = m; }
+          end = a;
+        }
+        sh.seg_end = end;
+      }
+      __syncthreads();
+      const int seg_hi = sh.seg_end;
+      const int nseg = seg_hi - seg_lo;
+      if (p.window > 0 && ARR) base = max_i64(base, (ARR[seg_lo] / p.window + 1) * p.window);
+
+      int L = 1;
+      if (geometric) {
+        L = sh.n_phases;
+        for (int q = tid; q <= L; q += T) {
+          int v;
+          if (q == 0) v = 0;
+          else if (q == L || family == KVS_GSA) v = nseg;
+          else {
+            const i64 t = sh.tau[q - 1];
+            int a = 0, b = nseg;
+            while (a < b) { const int m = (a + b) >> 1; if (K_ord[seg_lo + m] <= t) a = m + 1; else b = m; }
+            v = a;
+          }
+          sh.ent[q] = v;
+        }
+      } else if (tid == 0) {
+        const i64 tau = st.tau > 0 ? st.tau : static_cast<i64>(K_ord[seg_hi - 1]);   // largest key of the segment
+        i64 k = st.k;
+        if (k <= 0) k = sim ? M / (s_bar + tau) : (s_bar + tau <= M ? static_cast<i64>(max_parallelism32(static_cast<u32>(tau), static_cast<u32>(s_bar), static_cast<u32>(M))) : 0);
+        sh.tau[0] = static_cast<u32>(tau);
+        sh.k[0] = k < 1 ? 0u : static_cast<u32>(k);
+        sh.ent[0] = 0; sh.ent[1] = nseg;
+      }
+      if (carry) for (int i = tid; i < WARPS * MAXP; i += T) (&sh.cnt[0][0])[i] = 0;
+      __syncthreads();
+      if (!geometric && sh.k[0] < 1) { status = KVS_EVAL_INFEASIBLE; break; }
+
+      // ---- plan: participants, length and first round of every phase ----
+      const u32 Xc = static_cast<u32>(X);
+      // positions handled by one warp in the two counting passes (a multiple of 32)
+      const int per = (((nseg + WARPS - 1) / WARPS) + 31) & ~31;
+      const int x0 = min(nseg, warp * per), x1 = min(nseg, x0 + per);
+      if (carry) {
+        for (int x = x0 + lane; x < x1; x += 32) {
+          u32 v = static_cast<u32>(__ldg(O_ord + seg_lo + x));
+          if (est_class) { const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc); v = max(v, kc); }
+          atomicAdd(&sh.cnt[warp][class_of(sh.tau, L, v)], 1u);
+        }
+        __syncthreads();
+        if (tid < L) {
+          u32 h = 0;
+          for (int w = 0; w < WARPS; ++w) h += sh.cnt[w][tid];
+          sh.np[tid] = h;       // jobs that leave in phase tid
+        }
+        __syncthreads();
+      }
+      if (tid == 0) {
+        u32 gone = 0;
+        for (int q = 0; q < L; ++q) {
+          const u32 leave = carry ? sh.np[q] : static_cast<u32>(sh.ent[q + 1] - sh.ent[q]);
+          sh.np[q] = static_cast<u32>(sh.ent[q + 1]) - gone;
+          gone += leave;
+        }
+      }
+      __syncthreads();
+      if (tid < L) {
+        const u32 N = sh.np[tid], tau = sh.tau[tid], k = sh.k[tid];
+        i64 len = 0;
+        if (N > 0) len = (sim ? static_cast<i64>(ceil_div_u(N, k) - 1) * tau : static_cast<i64>(static_cast<u64>(N - 1) * tau / k)) + tau;
+        sh.plen[tid] = len;
+        // memory is kept modulo 2^32: the general kernel reports evaluations whose bound reaches that
+        if (walk && N > 0 && min_i64(N, static_cast<i64>(k) + 1) * (static_cast<i64>(stats.s_max) + tau) >= (static_cast<i64>(1) << 32))
+          sh.fallback = 1;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        i64 b = base, runs = sh.n_runs;
+        u64 tp = 0;
+        for (int q = 0; q < L; ++q) {
+          sh.taupre[q] = tp;
+          tp += sh.tau[q];
+          sh.pbase[q] = static_cast<u32>(b);
+          b += sh.plen[q];
+          runs += sh.np[q];
+          if (b >= TIME_LIMIT) { sh.fallback = 1; break; }
+        }
+        sh.taupre[L] = tp;
+        sh.base_next = b;
+        sh.n_runs = runs;
+      }
+      __syncthreads();
+      if (sh.fallback) { give_up = true; break; }
+
+      // ---- per-job results ----
+      if (!carry) {
+        // exactly one run per job; the rank is the position inside the class
+        const u32 tau0 = sh.tau[0];
+        for (int j = seg_lo + tid; j < seg_hi; j += T) {
+          const u32 oj = static_cast<u32>(__ldg(O_JOB + j));
+          const int pos = IPERM ? __ldg(IPERM + j) : j;
+          int ph = 0;
+          bool fin = true;
+          if (geometric) ph = class_of(sh.tau, L, oj);
+          else fin = oj <= tau0;
+          const u32 rank = static_cast<u32>(pos - seg_lo - sh.ent[ph]);
+          const u32 tau = sh.tau[ph], k = sh.k[ph];
+          const u32 stt = sh.pbase[ph] + (sim ? (rank / k) * tau : slot32(rank, tau, k));
+          const u32 d = fin ? oj : tau;
+          acc.steps += d;
+          acc.hmax = max(acc.hmax, stt + d);
+          int32_t start = -1, done = -1;
+          if (fin) {
+            start = static_cast<int32_t>(stt);
+            done = static_cast<int32_t>(stt + oj);
+            acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
+          } else {
+            ++acc.unfinished;
+          }
+          if (out_start) out_start[j] = start;
+          if (out_done) out_done[j] = done;
+        }
+      } else {
+        // ranks before each warp's segment: cnt[w][q] = #{positions in earlier segments that leave in phase q or later}
+        if (tid < WARPS) {
+          u32 run = 0;
+          for (int c = L - 1; c >= 0; --c) { run += sh.cnt[tid][c]; sh.cnt[tid][c] = run; }
+        }
+        __syncthreads();
+        if (tid < L) {
+          u32 run = 0;
+          for (int w = 0; w < WARPS; ++w) { const u32 t = sh.cnt[w][tid]; sh.cnt[w][tid] = run; run += t; }
+        }
+        __syncthreads();
+        u32 g0 = lane < L ? sh.cnt[warp][lane] : 0u;
+        u32 g1 = lane + 32 < L ? sh.cnt[warp][lane + 32] : 0u;
+        u32 g2 = lane + 64 < L ? sh.cnt[warp][lane + 64] : 0u;
+        for (int xb = x0; xb < x1; xb += 32) {
+          const int x = xb + lane;
+          const bool valid = x < x1;
+          u32 ov = 0;
+          int l = 0, f = 0;
+          if (valid) {
+            ov = static_cast<u32>(__ldg(O_ord + seg_lo + x));
+            u32 v = ov;
+            if (est_class) {
+              const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc);
+              f = class_of(sh.tau, L, kc);
+              v = max(v, kc);
+            }
+            l = class_of(sh.tau, L, v);
+          }
+          const u32 vm = __ballot_sync(0xffffffffu, valid);
+          const int nvalid = __popc(vm);
+          const int pmin = __reduce_min_sync(0xffffffffu, valid ? l : 0x7fffffff);
+          const int pmax = __reduce_max_sync(0xffffffffu, valid ? l : 0);
+          u32 rank = 0;
+          for (int q = pmin; q <= pmax; ++q) {
+            const u32 m = __ballot_sync(0xffffffffu, valid && l >= q);
+            const u32 gs = q < 32 ? g0 : (q < 64 ? g1 : g2);
+            const u32 g = __shfl_sync(0xffffffffu, gs, q & 31);
+            if (l == q) rank = g + __popc(m & lanemask_lt());
+            if (lane == (q & 31)) {
+              const u32 c = __popc(m);
+              if (q < 32) g0 += c; else if (q < 64) g1 += c; else g2 += c;
+            }
+          }
+          // every valid position counts for the phases before the smallest class seen
+          if (lane < pmin) g0 += nvalid;
+          if (lane + 32 < pmin) g1 += nvalid;
+          if (lane + 64 < pmin) g2 += nvalid;
+          if (valid) {
+            const u32 tau = sh.tau[l], k = sh.k[l];
+            const u32 stt = sh.pbase[l] + slot32(rank, tau, k);
+            acc.steps += ov + (sh.taupre[l] - sh.taupre[f]);
+            if (keyed) {
+              fin_start[seg_lo + x] = stt;
+            } else {
+              const int j = seg_lo + x;
+              const u32 done = stt + ov;
+              acc.hmax = max(acc.hmax, done);
+              acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
+              if (out_start) out_start[j] = static_cast<int32_t>(stt);
+              if (out_done) out_done[j] = static_cast<int32_t>(done);
+            }
+          }
+        }
+        if (keyed) {
+          __syncthreads();
+          for (int j = seg_lo + tid; j < seg_hi; j += T) {
+            const u32 oj = static_cast<u32>(__ldg(O_JOB + j));
+            const u32 stt = fin_start[__ldg(IPERM + j)];
+            const u32 done = stt + oj;
+            acc.hmax = max(acc.hmax, done);
+            acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
+            if (out_start) out_start[j] = static_cast<int32_t>(stt);
+            if (out_done) out_done[j] = static_cast<int32_t>(done);
+          }
+        }
+      }
+
+      // ---- memory profile ----
+      if (event_form) {
+        // SPS / SimS in exact key order with no profile wanted: the peak comes from the run ends
+        const i64* const ps = p.prefix_s + lo + st.instance + seg_lo;
+        const i64 N = nseg;
+        const i64 pr = (N + T - 1) / T;
+        const i64 i0 = min_i64(N, tid * pr), i1 = min_i64(N, i0 + pr);
+        u64 unused_flow = 0;
+        const i64 pk = sim ? sims_range_peak(O_ord + seg_lo, ps, N, sh.tau[0], sh.k[0], i0, i1, &unused_flow)
+                           : sps_range_peak(O_ord + seg_lo, ps, N, sh.tau[0], sh.k[0], i0, i1, &unused_flow);
+        acc.peak64 = max_i64(acc.peak64, pk);
+      } else if (walk) {
+        int C = 0;
+        uint2* cur = list0;
+        uint2* nxt = list1;
+        for (int ph = 0; ph < L; ++ph) {
+          const int N = static_cast<int>(sh.np[ph]);
+          if (N == 0) continue;
+          const int ent_lo = sh.ent[ph];
+          PhaseView P;
+          P.cur = cur; P.C = C;
+          P.S = S_ord + seg_lo + ent_lo; P.O = O_ord + seg_lo + ent_lo;
+          P.tau = sh.tau[ph]; P.k = sh.k[ph];
+          P.qt = P.tau / P.k; P.rt = P.tau - P.qt * P.k;
+          P.len = static_cast<u32>(sh.plen[ph]);
+          P.base = sh.pbase[ph];
+          const bool combine = sim && P.k >= 32;
+          const bool dense = !sim && P.tau < TILE && P.k >= 4 * P.tau;
+          // idle rounds before this phase (window release) hold nothing
+          if (prof_cap > 0)
+            for (i64 t = written_to + tid; t < P.base && t < prof_cap; t += T) prof[t] = 0;
+          // tile origins keep the profile stores 16-byte aligned
+          const int a0 = -static_cast<int>((prof_base + P.base) & 3);
+          u32 A_run = 0, B_run = 0;
+          int r_next = 0, buf = 0, C_next = 0;
+          // ranks that start before offset u: ceil(u*k/tau) (SPS) or ceil(u/tau)*k (SimS); the tile
+          // ends advance by TILE, so quotient and remainder are stepped
+          const u64 mult = sim ? 1 : static_cast<u64>(P.k);
+          const u64 utau = P.tau;
+          u64 cq, cr, dq, dr;
+          divmod_u(static_cast<u64>(a0 + TILE) * mult, utau, &cq, &cr);
+          divmod_u(static_cast<u64>(TILE) * mult, utau, &dq, &dr);
+          for (int u0 = a0; u0 < static_cast<int>(P.len); u0 += TILE) {
+            const int wlen = min(TILE, static_cast<int>(P.len) - u0);
+            int r_b = N;                          // the last tile takes every remaining rank
+            if (u0 + TILE < static_cast<int>(P.len)) {
+              const u64 rb64 = (cq + (cr > 0)) * (sim ? static_cast<u64>(P.k) : 1ull);
+              if (rb64 < static_cast<u64>(N)) r_b = static_cast<int>(rb64);
+            }
+            cq += dq; cr += dr;
+            if (cr >= utau) { cr -= utau; ++cq; }
+            if (sim) C_next = visit_runs<true, false>(sh, P, nxt, C_next, r_next, r_b, u0, buf, dense, combine);
+            else if (carry) C_next = visit_runs<false, true>(sh, P, nxt, C_next, r_next, r_b, u0, buf, dense, combine);
+            else C_next = visit_runs<false, false>(sh, P, nxt, C_next, r_next, r_b, u0, buf, dense, combine);
+            r_next = r_b;
+            if (P.tau > TILE) insert_far_ends(sh, P, sim, N, a0, u0, wlen, buf);
+            __syncthreads();
+            scan_tile(sh, buf, static_cast<i64>(P.base) + u0, wlen, P.base, A_run, B_run, acc.peak, prof, prof_cap);
+            buf ^= 1;
+          }
+          written_to = static_cast<i64>(P.base) + P.len;
+          __syncthreads();               // carry list complete before it is read as `cur`
+          uint2* tmp = cur; cur = nxt; nxt = tmp;
+          C = C_next;
+        }
+      }
+      base = sh.base_next;
+      seg_lo = seg_hi;
+    }
+
+    if (give_up) {
+      // left to the general kernel, which writes every output of this evaluation
+      if (tid == 0) p.slow_list[atomicAdd(p.slow_count, 1ull)] = e;
+      continue;
+    }
+
+    // ---- scalars ----
+    const i64 flow = static_cast<i64>(block_sum(acc.flow, reinterpret_cast<u64*>(sh.red64)));
+    const i64 steps = static_cast<i64>(block_sum(acc.steps, reinterpret_cast<u64*>(sh.red64)));
+    const i64 hmax = block_max(acc.hmax, sh.redA, 0u);
+    const int unfinished = block_sum(acc.unfinished, sh.red32);
+    const u32 peak32 = block_max(acc.peak, sh.redA, 0u);
+    const i64 peak = max_i64(static_cast<i64>(peak32), block_max(acc.peak64, sh.red64, static_cast<i64>(0)));
+    if (tid == 0) {
+      const bool skipped = (status & (KVS_EVAL_INFEASIBLE | KVS_EVAL_BAD_INPUT)) != 0;
+      if (!skipped && prof_cap > 0 && hmax > prof_cap) status |= KVS_EVAL_CAPACITY;   // capacity 0 = profile not wanted
+      const bool have_peak = p.do_profile && !skipped;
+      if (p.ev.peak) p.ev.peak[e] = have_peak ? peak : -1;
+      if (p.ev.flow) p.ev.flow[e] = flow;
+      if (p.ev.job_steps) p.ev.job_steps[e] = steps;
+      if (p.ev.horizon) p.ev.horizon[e] = hmax;
+      if (p.ev.n_unfinished) p.ev.n_unfinished[e] = unfinished;
+      if (p.ev.feasible) p.ev.feasible[e] = (have_peak && !(status & KVS_EVAL_RANGE) && peak <= M) ? 1 : 0;
+      if (p.ev.status) p.ev.status[e] = status;
+      if (p.out.n_runs) p.out.n_runs[e] = sh.n_runs;
+    }
+    (void)want32;
+  }
+}
+
+}  // namespace
+
+static size_t fused_smem_bytes() { return sizeof(FShared); }
+
+int kvs_fused_ctas_per_sm() {
+  int n = 0;
+  cudaFuncSetAttribute(k_fused_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes()));
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_fused_eval, KVS_EVAL_THREADS, fused_smem_bytes()) != cudaSuccess) n = 1;
+  return n < 1 ? 1 : n;
+}
+
+cudaError_t kvs_launch_fused(const BuildParams& p, int grid, cudaStream_t stream) {
+  if (p.P <= 0) return cudaSuccess;
+  cudaError_t err = cudaFuncSetAttribute(k_fused_eval, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(fused_smem_bytes()));
+  if (err != cudaSuccess) return err;
+  err = cudaMemsetAsync(p.counter, 0, 16, stream);   // work counter and length of the list of left-over evaluations
+  if (err != cudaSuccess) return err;
+  k_fused_eval<<<grid, KVS_EVAL_THREADS, fused_smem_bytes(), stream>>>(p);
+  return cudaGetLastError();
+}

@@ -60,6 +60,12 @@ struct BuildParams {
   // per-CTA carry lists: 2 * max_jobs entries each
   int32_t* lists;
   ull* counter;             // next evaluation to hand out (zeroed before each launch)
+  // The 32-bit fast kernel appends the evaluations it leaves to the general kernel here ...
+  i64* slow_list;
+  ull* slow_count;
+  // ... and the general kernel, when given a list, works through eval_list[0 .. *eval_count)
+  const i64* eval_list;
+  const ull* eval_count;
 };
 
 struct SortParams {
@@ -107,6 +113,8 @@ struct SweepParams {
 cudaError_t kvs_launch_sort(const SortParams& p, int grid, cudaStream_t stream);
 cudaError_t kvs_launch_build(const BuildParams& p, int grid, cudaStream_t stream);
 int kvs_build_ctas_per_sm();
+cudaError_t kvs_launch_fused(const BuildParams& p, int grid, cudaStream_t stream);
+int kvs_fused_ctas_per_sm();
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,
                               i64* prefix_o, cudaStream_t stream);

@@ -40,9 +40,19 @@ def check_batch(inst_cpu: Instances, settings: np.ndarray, *, window=0, want_pro
     dev = torch.device("cuda:0")
     if inst_gpu is None:
         inst_gpu = inst_cpu.to(dev)
-    res = scheduler().evaluate(inst_gpu, settings, want_jobs=True, want_profile=want_profile,
-                               want_runs=want_runs, window=window)
-    torch.cuda.synchronize()
+    # A call that asks for the explicit run list takes the general kernel, one that does not takes the
+    # 32-bit fast kernel: both are checked against the oracle.
+    variants = [want_runs] if not want_runs else [True, False]
+    steps = 0
+    for runs_wanted in variants:
+        res = scheduler().evaluate(inst_gpu, settings, want_jobs=True, want_profile=want_profile,
+                                   want_runs=runs_wanted, window=window)
+        torch.cuda.synchronize()
+        steps = _compare(res, inst_cpu, settings, window, want_profile, sample, f"{label} runs={int(runs_wanted)}")
+    return steps
+
+
+def _compare(res, inst_cpu, settings, window, want_profile, sample, label):
     g = {k: (v.cpu().numpy() if isinstance(v, torch.Tensor) else v) for k, v in vars(res).items() if k != "runs"}
     gruns = {k: v.cpu().numpy() for k, v in res.runs.items()} if res.runs else None
     P = settings.shape[0]
