@@ -61,7 +61,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.prefix_s = take(static_cast<size_t>(N + I) * 8);
   L.iperm = take(static_cast<size_t>(N) * 4);
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
-  L.lists = take(static_cast<size_t>(grid) * 2 * static_cast<size_t>(max_n) * 8);   // (s, o) pairs in the fast kernel
+  L.lists = take(static_cast<size_t>(grid) * static_cast<size_t>(KVS_CTA_SCRATCH(max_n)));
   L.fin_rank = take(static_cast<size_t>(grid) * static_cast<size_t>(max_n) * 4);
   L.counter = take(32);   // work counter of the fast kernel, length of its left-over list, work counter of the general kernel
   L.slow_list = take(static_cast<size_t>(P) * 8);

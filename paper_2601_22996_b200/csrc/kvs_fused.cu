@@ -140,174 +140,213 @@ __device__ __forceinline__ int slot(int e) { return ((((e >> 2) % VEC) * T + e /
 // Word of the round `rel` rounds after the origin of ring half `buf`, 0 <= rel < 2*TILE.
 __device__ __forceinline__ int ring(int buf, int rel) { return ((buf ^ (rel >= TILE ? 1 : 0)) * TILE) + slot(rel & (TILE - 1)); }
 
-__device__ __forceinline__ int block_count_scan(int v, int* red32, int* total) {
-  int incl = v;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, incl, d);
-    if (static_cast<int>(lane_id()) >= d) incl += y;
-  }
-  const int warp = threadIdx.x >> 5;
-  __syncthreads();
-  if (lane_id() == 31) red32[warp] = incl;
-  __syncthreads();
-  const int w = (lane_id() < WARPS) ? red32[lane_id()] : 0;
-  int wi = w;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, wi, d);
-    if (static_cast<int>(lane_id()) >= d) wi += y;
-  }
-  *total = __shfl_sync(0xffffffffu, wi, 31);
-  return __shfl_sync(0xffffffffu, wi - w, warp) + (incl - v);
-}
-
-// One phase as the run visit sees it.  Participants in rank order: `C` carried (s, o) pairs in
-// `cur`, then the positions src_lo .. of the instance's schedule order.
+// One phase as the run visit sees it.  Positions are relative to the window, in schedule order.
+// Exact keys: the participants are the positions [x_lo, x_hi) and the rank is the offset from x_lo.
+// Carried jobs (FILTER): position x < x_hi takes part iff its leaving class cls[x] >= ph, and the
+// rank table G[seg * L + ph] holds the number of such positions before segment `seg` (SEG positions
+// each), so a warp can start at any segment without looking at the ones before it.
 struct PhaseView {
-  const uint2* cur;
   const int32_t* S;
   const int32_t* O;
-  int C;
+  const unsigned char* cls;
+  const u32* G;
+  int L, ph, nsegs;
+  int x_lo, x_hi;
   u32 tau, k, qt, rt;     // tau = qt*k + rt
   u32 len;                // rounds of the phase
   u32 base;               // its first round
 };
 
+constexpr int SEG = 256;  // positions per warp step: 8 consecutive positions per lane
+
+// The 8 positions of one lane in segment `seg`: bit j of `bits` is set if position xb + j takes part,
+// and those positions have the consecutive ranks r_first, r_first + 1, ...
+struct LaneGroup { u32 bits; int r_first; int xb; };
+
+template <bool FILTER>
+__device__ __forceinline__ LaneGroup lane_group(const PhaseView& P, int seg) {
+  LaneGroup g;
+  const int lane = lane_id();
+  if (FILTER) {
+    g.xb = seg * SEG + 8 * lane;
+    const uint2 cw = *reinterpret_cast<const uint2*>(P.cls + g.xb);
+    const int room = P.x_hi - g.xb;                        // positions of this lane below x_hi
+    const u32 lim = room >= 8 ? 0xffu : (room > 0 ? (1u << room) - 1u : 0u);
+    u32 bits = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const u32 c = ((j < 4 ? cw.x : cw.y) >> (8 * (j & 3))) & 255u;
+      if (c >= static_cast<u32>(P.ph)) bits |= 1u << j;
+    }
+    g.bits = bits & lim;
+    int incl = __popc(g.bits);
+    const int cnt = incl;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    g.r_first = static_cast<int>(P.G[seg * P.L + P.ph]) + incl - cnt;
+  } else {
+    g.r_first = seg * SEG + 8 * lane;
+    g.xb = P.x_lo + g.r_first;
+    const int room = P.x_hi - g.xb;
+    g.bits = room >= 8 ? 0xffu : (room > 0 ? (1u << room) - 1u : 0u);
+  }
+  return g;
+}
+
+// Segments that hold the ranks [ra, rb) of the phase.
+template <bool FILTER>
+__device__ __forceinline__ void segment_range(const PhaseView& P, int ra, int rb, int* seg_a, int* seg_b) {
+  if (FILTER) {
+    // G[.][ph] is nondecreasing over the nsegs + 1 rows; last row = number of participants
+    int a = 0, b = P.nsegs;               // largest seg with G[seg] <= ra
+    while (a < b) { const int m = (a + b + 1) >> 1; if (static_cast<int>(P.G[m * P.L + P.ph]) <= ra) a = m; else b = m - 1; }
+    *seg_a = a;
+    a = 0; b = P.nsegs;                   // smallest seg with G[seg] >= rb
+    while (a < b) { const int m = (a + b) >> 1; if (static_cast<int>(P.G[m * P.L + P.ph]) >= rb) b = m; else a = m + 1; }
+    *seg_b = a;
+  } else {
+    *seg_a = ra / SEG;
+    *seg_b = (rb + SEG - 1) / SEG;
+  }
+}
+
 // Visits ranks [ra, rb), all of which start inside the tile whose origin is `trel` rounds after
 // the phase's first round (trel may be slightly negative) and whose ring half is `buf`: adds the
-// two events of every run and appends the killed jobs to `nxt`.  Returns the new length of `nxt`.
-template <bool SIM, bool CARRY>
-__device__ __forceinline__ int visit_runs(FShared& sh, const PhaseView& P, uint2* nxt, int C_next,
-                                          int ra, int rb, int trel, int buf, bool dense, bool combine) {
-  const int tid = threadIdx.x;
+// two events of every run.  Warps take segments in turn; nothing is written to global memory and
+// no block-wide barrier is needed.
+template <bool SIM, bool FILTER>
+__device__ __forceinline__ void visit_runs(FShared& sh, const PhaseView& P, int ra, int rb, int trel, int buf,
+                                           bool dense, bool combine) {
+  if (ra >= rb) return;
   u32* const dA = reinterpret_cast<u32*>(sh.dA);
   u32* const dB = reinterpret_cast<u32*>(sh.dB);
   const u32 tau = P.tau, k = P.k;
-  for (int c0 = ra; c0 < rb;) {
-    const int left = rb - c0;
-    const int rpt = left > 2 * T ? RPT : (left > T ? 2 : 1);
-    const int r_first = c0 + tid * rpt;
-    c0 += T * rpt;
-    uint2 keep[RPT];
-    u32 cmask = 0;
-    if (r_first - static_cast<int>(lane_id()) * rpt < rb) {   // warps past the end of the range skip the visit
-      u32 s_[RPT], o_[RPT];
-      bool on[RPT];
+  const int warp = threadIdx.x >> 5;
+  int seg_a, seg_b;
+  segment_range<FILTER>(P, ra, rb, &seg_a, &seg_b);
+  for (int seg = seg_a + warp; seg < seg_b; seg += WARPS) {
+    const LaneGroup g = lane_group<FILTER>(P, seg);
+    // of this lane's participants, entries [skip, skip + take) have ranks inside [ra, rb)
+    const int cnt = __popc(g.bits);
+    const int skip = max(0, ra - g.r_first);
+    const int take = min(cnt, rb - g.r_first) - skip;
+    if (__ballot_sync(0xffffffffu, take > 0) == 0) continue;
+    u32 s_[8], o_[8];
 #pragma unroll
-      for (int j = 0; j < RPT; ++j) {
-        const int r = r_first + j;
-        on[j] = j < rpt && r < rb;
-        s_[j] = 0; o_[j] = 0;
-        if (on[j]) {
-          if (r < P.C) { const uint2 e = P.cur[r]; s_[j] = e.x; o_[j] = e.y; }
-          else { s_[j] = static_cast<u32>(__ldg(P.S + (r - P.C))); o_[j] = static_cast<u32>(__ldg(P.O + (r - P.C))); }
-        }
-      }
-      u32 q = 0, rem = 0;      // start offset of the current rank inside the phase and its remainder
-      if (on[0]) {
-        if (SIM) {
-          const u32 b = static_cast<u32>(r_first) / k;
-          q = b * tau;
-          rem = static_cast<u32>(r_first) - b * k;
-        } else {
-          u64 dq_, dr_;
-          divmod_u(static_cast<u64>(r_first) * tau, k, &dq_, &dr_);
-          q = static_cast<u32>(dq_);
-          rem = static_cast<u32>(dr_);
-        }
-      }
-      // Dense phases (several runs start per round): the runs of a lane that start in the round of
-      // its first run are summed in registers, then equal rounds - contiguous lanes, because
-      // consecutive ranks start in nondecreasing rounds - are summed across the warp with a
-      // segmented scan, and one lane per round issues the atomics.  Runs that hold their whole
-      // slot end together (start + tau), so their end events are combined the same way.
-      const bool dn = !SIM && dense;
-      int seg = 0x7fffffff;
-      u32 seg_all = 0, seg_full = 0, seg_cnt = 0;
-#pragma unroll
-      for (int j = 0; j < RPT; ++j) {
-        int sidx = -1, eidx = -1;
-        u32 c = 0;
-        if (on[j]) {
-          const u32 oi = o_[j];
-          const u32 d = oi < tau ? oi : tau;
-          if (CARRY && oi > tau) { keep[j] = make_uint2(s_[j], oi); cmask |= 1u << j; }
-          c = s_[j] + 1u - P.base - q;                          // tokens(t) = c + t while active
-          const int srel = static_cast<int>(q) - trel;
-          sidx = ring(buf, srel);
-          if (q + d < P.len) {                                   // an end at the phase end is never read
-            const u32 erel = static_cast<u32>(srel) + d;
-            if (erel < 2u * TILE) eidx = ring(buf, static_cast<int>(erel));
-          }
-          if (dn) {
-            if (seg == 0x7fffffff) seg = srel;
-            if (srel == seg) {
-              seg_all += c; seg_cnt += 1u;
-              sidx = -1;
-              if (d == tau) { seg_full += c; seg_cnt += 1u << 16; eidx = -1; }
-            }
-          }
-          if (SIM) { if (++rem == k) { rem = 0; q += tau; } }
-          else { rem += P.rt; q += P.qt; if (rem >= k) { rem -= k; ++q; } }
-        }
-        if (SIM && combine) {
-          // whole simultaneous batches hit one word: sum equal targets inside the warp first
-          const u32 ps = __match_any_sync(0xffffffffu, sidx);
-          if (sidx >= 0) {
-            const u32 cs = __reduce_add_sync(ps, c);
-            if ((ps & lanemask_lt()) == 0) { atomicAdd(&dA[sidx], cs); atomicAdd(&dB[sidx], static_cast<u32>(__popc(ps))); }
-          }
-          const u32 pe = __match_any_sync(0xffffffffu, eidx);
-          if (eidx >= 0) {
-            const u32 ce = __reduce_add_sync(pe, c);
-            if ((pe & lanemask_lt()) == 0) { atomicAdd(&dA[eidx], 0u - ce); atomicAdd(&dB[eidx], 0u - static_cast<u32>(__popc(pe))); }
-          }
-        } else {
-          if (sidx >= 0) { atomicAdd(&dA[sidx], c); atomicAdd(&dB[sidx], 1u); }
-          if (eidx >= 0) { atomicAdd(&dA[eidx], 0u - c); atomicAdd(&dB[eidx], 0xffffffffu); }
-        }
-      }
-      if (dn) {
-        int key = seg;
-        u32 va = seg_all, vf = seg_full, vn = seg_cnt;
-#pragma unroll
-        for (int dd = 1; dd < 32; dd <<= 1) {
-          const int kk = __shfl_up_sync(0xffffffffu, key, dd);
-          const u32 ya = __shfl_up_sync(0xffffffffu, va, dd), yf = __shfl_up_sync(0xffffffffu, vf, dd);
-          const u32 yn = __shfl_up_sync(0xffffffffu, vn, dd);
-          if (static_cast<int>(lane_id()) >= dd && kk == key) { va += ya; vf += yf; vn += yn; }
-        }
-        const int next_key = __shfl_down_sync(0xffffffffu, key, 1);
-        if (key != 0x7fffffff && (lane_id() == 31 || next_key != key)) {   // last lane of its round
-          const int si = ring(buf, key);
-          atomicAdd(&dA[si], va);
-          atomicAdd(&dB[si], vn & 0xffffu);
-          const u32 n_full = vn >> 16;
-          // start offset of this round inside the phase: key + trel
-          if (n_full && static_cast<u32>(key + trel) + tau < P.len) {
-            const int ei = ring(buf, key + static_cast<int>(tau));          // tau < TILE in dense phases
-            atomicAdd(&dA[ei], 0u - vf);
-            atomicAdd(&dB[ei], 0u - n_full);
-          }
-        }
+    for (int j = 0; j < 8; ++j) {
+      s_[j] = 0; o_[j] = 0;
+      if (take > 0 && (g.bits >> j & 1u)) {
+        s_[j] = static_cast<u32>(__ldg(P.S + g.xb + j));
+        o_[j] = static_cast<u32>(__ldg(P.O + g.xb + j));
       }
     }
-    if (CARRY) {
-      int total;
-      int off = C_next + block_count_scan(__popc(cmask), sh.red32, &total);
+    u32 q = 0, rem = 0;      // start offset of the current rank inside the phase and its remainder
+    if (take > 0) {
+      const u32 r0 = static_cast<u32>(g.r_first + skip);
+      if (SIM) {
+        const u32 b = r0 / k;
+        q = b * tau;
+        rem = r0 - b * k;
+      } else {
+        u64 dq_, dr_;
+        divmod_u(static_cast<u64>(r0) * tau, k, &dq_, &dr_);
+        q = static_cast<u32>(dq_);
+        rem = static_cast<u32>(dr_);
+      }
+    }
+    // Dense phases (several runs start per round): the runs of a lane that start in the round of
+    // its first run are summed in registers, then equal rounds - contiguous lanes, because
+    // consecutive ranks start in nondecreasing rounds - are summed across the warp with a
+    // segmented scan, and one lane per round issues the atomics.  Runs that hold their whole
+    // slot end together (start + tau), so their end events are combined the same way.
+    const bool dn = !SIM && dense;
+    int seg_key = 0x7fffffff;
+    u32 seg_all = 0, seg_full = 0, seg_cnt = 0;
+    int idx = 0;             // index among this lane's participants
 #pragma unroll
-      for (int j = 0; j < RPT; ++j)
-        if (cmask >> j & 1u) nxt[off++] = keep[j];
-      C_next += total;
+    for (int j = 0; j < 8; ++j) {
+      int sidx = -1, eidx = -1;
+      u32 c = 0;
+      const bool part = (g.bits >> j & 1u) != 0;
+      const bool on = part && idx >= skip && idx < skip + take;
+      if (part) ++idx;
+      if (on) {
+        const u32 oi = o_[j];
+        const u32 d = oi < tau ? oi : tau;
+        c = s_[j] + 1u - P.base - q;                          // tokens(t) = c + t while active
+        const int srel = static_cast<int>(q) - trel;
+        sidx = ring(buf, srel);
+        if (q + d < P.len) {                                   // an end at the phase end is never read
+          const u32 erel = static_cast<u32>(srel) + d;
+          if (erel < 2u * TILE) eidx = ring(buf, static_cast<int>(erel));
+        }
+        if (dn) {
+          if (seg_key == 0x7fffffff) seg_key = srel;
+          if (srel == seg_key) {
+            seg_all += c; seg_cnt += 1u;
+            sidx = -1;
+            if (d == tau) { seg_full += c; seg_cnt += 1u << 16; eidx = -1; }
+          }
+        }
+        if (SIM) { if (++rem == k) { rem = 0; q += tau; } }
+        else { rem += P.rt; q += P.qt; if (rem >= k) { rem -= k; ++q; } }
+      }
+      if (SIM && combine) {
+        // whole simultaneous batches hit one word: sum equal targets inside the warp first
+        const u32 ps = __match_any_sync(0xffffffffu, sidx);
+        if (sidx >= 0) {
+          const u32 cs = __reduce_add_sync(ps, c);
+          if ((ps & lanemask_lt()) == 0) { atomicAdd(&dA[sidx], cs); atomicAdd(&dB[sidx], static_cast<u32>(__popc(ps))); }
+        }
+        const u32 pe = __match_any_sync(0xffffffffu, eidx);
+        if (eidx >= 0) {
+          const u32 ce = __reduce_add_sync(pe, c);
+          if ((pe & lanemask_lt()) == 0) { atomicAdd(&dA[eidx], 0u - ce); atomicAdd(&dB[eidx], 0u - static_cast<u32>(__popc(pe))); }
+        }
+      } else {
+        if (sidx >= 0) { atomicAdd(&dA[sidx], c); atomicAdd(&dB[sidx], 1u); }
+        if (eidx >= 0) { atomicAdd(&dA[eidx], 0u - c); atomicAdd(&dB[eidx], 0xffffffffu); }
+      }
+    }
+    if (dn) {
+      // a lane without runs takes the round of the nearest lane before it that has some, so that
+      // equal rounds stay contiguous for the segmented scan
+      const u32 has = __ballot_sync(0xffffffffu, seg_key != 0x7fffffff);
+      const u32 before = has & lanemask_lt();
+      const int src = (seg_key == 0x7fffffff && before) ? 31 - __clz(before) : static_cast<int>(lane_id());
+      int key = __shfl_sync(0xffffffffu, seg_key, src);
+      u32 va = seg_all, vf = seg_full, vn = seg_cnt;
+#pragma unroll
+      for (int dd = 1; dd < 32; dd <<= 1) {
+        const int kk = __shfl_up_sync(0xffffffffu, key, dd);
+        const u32 ya = __shfl_up_sync(0xffffffffu, va, dd), yf = __shfl_up_sync(0xffffffffu, vf, dd);
+        const u32 yn = __shfl_up_sync(0xffffffffu, vn, dd);
+        if (static_cast<int>(lane_id()) >= dd && kk == key) { va += ya; vf += yf; vn += yn; }
+      }
+      const int next_key = __shfl_down_sync(0xffffffffu, key, 1);
+      if (key != 0x7fffffff && (lane_id() == 31 || next_key != key)) {   // last lane of its round
+        const int si = ring(buf, key);
+        atomicAdd(&dA[si], va);
+        atomicAdd(&dB[si], vn & 0xffffu);
+        const u32 n_full = vn >> 16;
+        // start offset of this round inside the phase: key + trel
+        if (n_full && static_cast<u32>(key + trel) + tau < P.len) {
+          const int ei = ring(buf, key + static_cast<int>(tau));          // tau < TILE in dense phases
+          atomicAdd(&dA[ei], 0u - vf);
+          atomicAdd(&dB[ei], 0u - n_full);
+        }
+      }
     }
   }
-  return C_next;
 }
 
 // Slices longer than a tile: ends that land two or more tiles after the run's start were not
 // inserted when the run was visited; pick them up when their tile comes.  u0 = offset of this
 // tile's origin inside the phase, a0 = the same for the phase's first tile (0 or slightly negative).
+template <bool FILTER>
 __device__ __forceinline__ void insert_far_ends(FShared& sh, const PhaseView& P, bool sim, int N, int a0, int u0,
                                                 int wlen, int buf) {
   if (u0 <= TILE) return;
@@ -316,16 +355,23 @@ __device__ __forceinline__ void insert_far_ends(FShared& sh, const PhaseView& P,
   if (sim) { r_lo = ceil_div_u(lo, P.tau) * P.k; r_hi = ceil_div_u(hi, P.tau) * P.k; }
   else { r_lo = ceil_div_u(static_cast<u64>(lo) * P.k, P.tau); r_hi = ceil_div_u(static_cast<u64>(hi) * P.k, P.tau); }
   if (r_hi > N) r_hi = N;
+  if (r_lo >= r_hi) return;
+  const int ra = static_cast<int>(r_lo), rb = static_cast<int>(r_hi);
   u32* const dA = reinterpret_cast<u32*>(sh.dA);
   u32* const dB = reinterpret_cast<u32*>(sh.dB);
-  for (i64 r0 = r_lo; r0 < r_hi; r0 += T) {
-    const i64 rr = r0 + threadIdx.x;
-    if (rr < r_hi) {
-      const int r = static_cast<int>(rr);
-      u32 si, oi;
-      if (r < P.C) { const uint2 e = P.cur[r]; si = e.x; oi = e.y; }
-      else { si = static_cast<u32>(__ldg(P.S + (r - P.C))); oi = static_cast<u32>(__ldg(P.O + (r - P.C))); }
-      const u32 q = sim ? (static_cast<u32>(r) / P.k) * P.tau : slot32(static_cast<u32>(r), P.tau, P.k);
+  const int warp = threadIdx.x >> 5;
+  int seg_a, seg_b;
+  segment_range<FILTER>(P, ra, rb, &seg_a, &seg_b);
+  for (int seg = seg_a + warp; seg < seg_b; seg += WARPS) {
+    const LaneGroup g = lane_group<FILTER>(P, seg);
+    int r = g.r_first;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (!(g.bits >> j & 1u)) continue;
+      const int rr = r++;
+      if (rr < ra || rr >= rb) continue;
+      const u32 si = static_cast<u32>(__ldg(P.S + g.xb + j)), oi = static_cast<u32>(__ldg(P.O + g.xb + j));
+      const u32 q = sim ? (static_cast<u32>(rr) / P.k) * P.tau : slot32(static_cast<u32>(rr), P.tau, P.k);
       const u32 end = q + (oi < P.tau ? oi : P.tau);
       const int ts = a0 + ((static_cast<int>(q) - a0) / TILE) * TILE;   // origin of the tile the run started in
       if (static_cast<int>(end) >= ts + 2 * TILE && static_cast<int>(end) >= u0 && static_cast<int>(end) < u0 + wlen && end < P.len) {
@@ -336,6 +382,16 @@ __device__ __forceinline__ void insert_far_ends(FShared& sh, const PhaseView& P,
       }
     }
   }
+}
+
+// inclusive suffix sum across the lanes of a warp
+__device__ __forceinline__ u32 warp_suffix(u32 v) {
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 y = __shfl_down_sync(0xffffffffu, v, d);
+    if (static_cast<int>(lane_id()) + d < 32) v += y;
+  }
+  return v;
 }
 
 // Prefix-sums one tile of the ring, turns it into memory(t), reduces the peak, stores the profile
@@ -414,8 +470,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
   extern __shared__ __align__(16) unsigned char smem_raw[];
   FShared& sh = *reinterpret_cast<FShared*>(smem_raw);
   const int tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
-  uint2* const list0 = reinterpret_cast<uint2*>(p.lists) + static_cast<i64>(blockIdx.x) * 2 * p.max_jobs;
-  uint2* const list1 = list0 + p.max_jobs;
+  // per-CTA scratch: class bytes of the current window (padded to whole segments), then the rank table
+  unsigned char* const cls = reinterpret_cast<unsigned char*>(p.lists) + static_cast<i64>(blockIdx.x) * KVS_CTA_SCRATCH(p.max_jobs);
+  u32* const G = reinterpret_cast<u32*>(cls + ((p.max_jobs + SEG + 15) & ~static_cast<i64>(15)));
   u32* const fin_start = reinterpret_cast<u32*>(p.fin_rank) + static_cast<i64>(blockIdx.x) * p.max_jobs;
   {
     const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -523,34 +580,75 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
 
       // ---- plan: participants, length and first round of every phase ----
       const u32 Xc = static_cast<u32>(X);
-      // positions handled by one warp in the two counting passes (a multiple of 32)
-      const int per = (((nseg + WARPS - 1) / WARPS) + 31) & ~31;
-      const int x0 = min(nseg, warp * per), x1 = min(nseg, x0 + per);
+      const int nsegs = (nseg + SEG - 1) / SEG;
       if (carry) {
-        for (int x = x0 + lane; x < x1; x += 32) {
-          u32 v = static_cast<u32>(__ldg(O_ord + seg_lo + x));
-          if (est_class) { const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc); v = max(v, kc); }
-          atomicAdd(&sh.cnt[warp][class_of(sh.tau, L, v)], 1u);
+        // leaving class of every position, and per segment the number of positions that leave in
+        // phase q or later (row `seg` of the table, not yet summed over the segments before it)
+        for (int seg = warp; seg < nsegs; seg += WARPS) {
+          const int xb = seg * SEG + 8 * lane;
+          u32 w0 = 0, w1 = 0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int x = xb + j;
+            u32 c = 0;
+            if (x < nseg) {
+              u32 v = static_cast<u32>(__ldg(O_ord + seg_lo + x));
+              if (est_class) { const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc); v = max(v, kc); }
+              c = static_cast<u32>(class_of(sh.tau, L, v));
+              atomicAdd(&sh.cnt[warp][c], 1u);
+            }
+            if (j < 4) w0 |= c << (8 * j); else w1 |= c << (8 * (j - 4));
+          }
+          *reinterpret_cast<uint2*>(cls + xb) = make_uint2(w0, w1);
+          __syncwarp();
+          u32 h0 = lane < L ? sh.cnt[warp][lane] : 0u;
+          u32 h1 = lane + 32 < L ? sh.cnt[warp][lane + 32] : 0u;
+          u32 h2 = lane + 64 < L ? sh.cnt[warp][lane + 64] : 0u;
+          if (lane < L) sh.cnt[warp][lane] = 0;
+          if (lane + 32 < L) sh.cnt[warp][lane + 32] = 0;
+          if (lane + 64 < L) sh.cnt[warp][lane + 64] = 0;
+          h2 = warp_suffix(h2);
+          h1 = warp_suffix(h1) + __shfl_sync(0xffffffffu, h2, 0);
+          h0 = warp_suffix(h0) + __shfl_sync(0xffffffffu, h1, 0);
+          if (lane < L) G[seg * L + lane] = h0;
+          if (lane + 32 < L) G[seg * L + lane + 32] = h1;
+          if (lane + 64 < L) G[seg * L + lane + 64] = h2;
+          __syncwarp();
         }
         __syncthreads();
-        if (tid < L) {
-          u32 h = 0;
-          for (int w = 0; w < WARPS; ++w) h += sh.cnt[w][tid];
-          sh.np[tid] = h;       // jobs that leave in phase tid
+        // exclusive sums over the segments; row nsegs = totals
+        const int rpw = (nsegs + WARPS - 1) / WARPS;
+        const int sa = min(nsegs, warp * rpw), sb = min(nsegs, sa + rpw);
+        u32 a0 = 0, a1 = 0, a2 = 0;
+        for (int seg = sa; seg < sb; ++seg) {
+          if (lane < L) a0 += G[seg * L + lane];
+          if (lane + 32 < L) a1 += G[seg * L + lane + 32];
+          if (lane + 64 < L) a2 += G[seg * L + lane + 64];
+        }
+        sh.cnt[warp][lane] = a0; sh.cnt[warp][lane + 32] = a1; sh.cnt[warp][lane + 64] = a2;
+        __syncthreads();
+        u32 r0 = 0, r1 = 0, r2 = 0;
+        for (int w = 0; w < warp; ++w) { r0 += sh.cnt[w][lane]; r1 += sh.cnt[w][lane + 32]; r2 += sh.cnt[w][lane + 64]; }
+        for (int seg = sa; seg < sb; ++seg) {
+          if (lane < L) { const u32 t = G[seg * L + lane]; G[seg * L + lane] = r0; r0 += t; }
+          if (lane + 32 < L) { const u32 t = G[seg * L + lane + 32]; G[seg * L + lane + 32] = r1; r1 += t; }
+          if (lane + 64 < L) { const u32 t = G[seg * L + lane + 64]; G[seg * L + lane + 64] = r2; r2 += t; }
+        }
+        if (warp == WARPS - 1) {
+          // positions that leave in phase q or later: all of them take part in q once they have entered
+          if (lane < L) { G[nsegs * L + lane] = r0; sh.np[lane] = r0; }
+          if (lane + 32 < L) { G[nsegs * L + lane + 32] = r1; sh.np[lane + 32] = r1; }
+          if (lane + 64 < L) { G[nsegs * L + lane + 64] = r2; sh.np[lane + 64] = r2; }
         }
         __syncthreads();
+        for (int i = tid; i < WARPS * MAXP; i += T) (&sh.cnt[0][0])[i] = 0;
       }
-      if (tid == 0) {
-        u32 gone = 0;
-        for (int q = 0; q < L; ++q) {
-          const u32 leave = carry ? sh.np[q] : static_cast<u32>(sh.ent[q + 1] - sh.ent[q]);
-          sh.np[q] = static_cast<u32>(sh.ent[q + 1]) - gone;
-          gone += leave;
-        }
-      }
-      __syncthreads();
       if (tid < L) {
-        const u32 N = sh.np[tid], tau = sh.tau[tid], k = sh.k[tid];
+        // entered by phase tid: positions below ent[tid + 1]; of those, the ones that leave in tid or later
+        const u32 N = carry ? static_cast<u32>(sh.ent[tid + 1]) - static_cast<u32>(nseg) + sh.np[tid]
+                            : static_cast<u32>(sh.ent[tid + 1] - sh.ent[tid]);
+        sh.np[tid] = N;
+        const u32 tau = sh.tau[tid], k = sh.k[tid];
         i64 len = 0;
         if (N > 0) len = (sim ? static_cast<i64>(ceil_div_u(N, k) - 1) * tau : static_cast<i64>(static_cast<u64>(N - 1) * tau / k)) + tau;
         sh.plen[tid] = len;
@@ -606,34 +704,22 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           if (out_done) out_done[j] = done;
         }
       } else {
-        // ranks before each warp's segment: cnt[w][q] = #{positions in earlier segments that leave in phase q or later}
-        if (tid < WARPS) {
-          u32 run = 0;
-          for (int c = L - 1; c >= 0; --c) { run += sh.cnt[tid][c]; sh.cnt[tid][c] = run; }
-        }
-        __syncthreads();
-        if (tid < L) {
-          u32 run = 0;
-          for (int w = 0; w < WARPS; ++w) { const u32 t = sh.cnt[w][tid]; sh.cnt[w][tid] = run; run += t; }
-        }
-        __syncthreads();
-        u32 g0 = lane < L ? sh.cnt[warp][lane] : 0u;
-        u32 g1 = lane + 32 < L ? sh.cnt[warp][lane + 32] : 0u;
-        u32 g2 = lane + 64 < L ? sh.cnt[warp][lane + 64] : 0u;
-        for (int xb = x0; xb < x1; xb += 32) {
+        // The rank of a job in the phase that completes it = positions before it that leave in that
+        // phase or later: the table gives the count before the segment, ballots the rest.
+        for (int seg = warp; seg < nsegs; seg += WARPS) {
+        u32 g0 = lane < L ? G[seg * L + lane] : 0u;
+        u32 g1 = lane + 32 < L ? G[seg * L + lane + 32] : 0u;
+        u32 g2 = lane + 64 < L ? G[seg * L + lane + 64] : 0u;
+        const int x1 = min(nseg, (seg + 1) * SEG);
+        for (int xb = seg * SEG; xb < x1; xb += 32) {
           const int x = xb + lane;
           const bool valid = x < x1;
           u32 ov = 0;
           int l = 0, f = 0;
           if (valid) {
             ov = static_cast<u32>(__ldg(O_ord + seg_lo + x));
-            u32 v = ov;
-            if (est_class) {
-              const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc);
-              f = class_of(sh.tau, L, kc);
-              v = max(v, kc);
-            }
-            l = class_of(sh.tau, L, v);
+            if (est_class) f = class_of(sh.tau, L, min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc));
+            l = cls[x];
           }
           const u32 vm = __ballot_sync(0xffffffffu, valid);
           const int nvalid = __popc(vm);
@@ -670,6 +756,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             }
           }
         }
+        }
         if (keyed) {
           __syncthreads();
           for (int j = seg_lo + tid; j < seg_hi; j += T) {
@@ -696,16 +783,14 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
                            : sps_range_peak(O_ord + seg_lo, ps, N, sh.tau[0], sh.k[0], i0, i1, &unused_flow);
         acc.peak64 = max_i64(acc.peak64, pk);
       } else if (walk) {
-        int C = 0;
-        uint2* cur = list0;
-        uint2* nxt = list1;
         for (int ph = 0; ph < L; ++ph) {
           const int N = static_cast<int>(sh.np[ph]);
           if (N == 0) continue;
-          const int ent_lo = sh.ent[ph];
           PhaseView P;
-          P.cur = cur; P.C = C;
-          P.S = S_ord + seg_lo + ent_lo; P.O = O_ord + seg_lo + ent_lo;
+          P.S = S_ord + seg_lo; P.O = O_ord + seg_lo;
+          P.cls = cls; P.G = G; P.L = L; P.ph = ph; P.nsegs = nsegs;
+          P.x_lo = carry ? 0 : sh.ent[ph];
+          P.x_hi = sh.ent[ph + 1];
           P.tau = sh.tau[ph]; P.k = sh.k[ph];
           P.qt = P.tau / P.k; P.rt = P.tau - P.qt * P.k;
           P.len = static_cast<u32>(sh.plen[ph]);
@@ -718,7 +803,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           // tile origins keep the profile stores 16-byte aligned
           const int a0 = -static_cast<int>((prof_base + P.base) & 3);
           u32 A_run = 0, B_run = 0;
-          int r_next = 0, buf = 0, C_next = 0;
+          int r_next = 0, buf = 0;
           // ranks that start before offset u: ceil(u*k/tau) (SPS) or ceil(u/tau)*k (SimS); the tile
           // ends advance by TILE, so quotient and remainder are stepped
           const u64 mult = sim ? 1 : static_cast<u64>(P.k);
@@ -735,19 +820,19 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             }
             cq += dq; cr += dr;
             if (cr >= utau) { cr -= utau; ++cq; }
-            if (sim) C_next = visit_runs<true, false>(sh, P, nxt, C_next, r_next, r_b, u0, buf, dense, combine);
-            else if (carry) C_next = visit_runs<false, true>(sh, P, nxt, C_next, r_next, r_b, u0, buf, dense, combine);
-            else C_next = visit_runs<false, false>(sh, P, nxt, C_next, r_next, r_b, u0, buf, dense, combine);
+            if (sim) visit_runs<true, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
+            else if (carry) visit_runs<false, true>(sh, P, r_next, r_b, u0, buf, dense, combine);
+            else visit_runs<false, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             r_next = r_b;
-            if (P.tau > TILE) insert_far_ends(sh, P, sim, N, a0, u0, wlen, buf);
+            if (P.tau > TILE) {
+              if (carry) insert_far_ends<true>(sh, P, sim, N, a0, u0, wlen, buf);
+              else insert_far_ends<false>(sh, P, sim, N, a0, u0, wlen, buf);
+            }
             __syncthreads();
             scan_tile(sh, buf, static_cast<i64>(P.base) + u0, wlen, P.base, A_run, B_run, acc.peak, prof, prof_cap);
             buf ^= 1;
           }
           written_to = static_cast<i64>(P.base) + P.len;
-          __syncthreads();               // carry list complete before it is read as `cur`
-          uint2* tmp = cur; cur = nxt; nxt = tmp;
-          C = C_next;
         }
       }
       base = sh.base_next;
