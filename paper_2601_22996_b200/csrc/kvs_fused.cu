@@ -127,6 +127,14 @@ __device__ __forceinline__ int class_of(const u32* tau, int L, u32 v) {
   return a;
 }
 
+// The same for the ladder of alpha = 2, tau_p = X >> (ell - p) with ell = floor(log2 X): the largest
+// shift j with (X >> j) >= v is the difference of the bit lengths, or one less.  1 <= v <= X.
+__device__ __forceinline__ int class_pow2(u32 X, u32 v) {
+  const int j0 = __clz(v) - __clz(X);
+  const int j = (X >> j0) >= v ? j0 : j0 - 1;
+  return (31 - __clz(X)) - j;
+}
+
 // floor(r * tau / k) for r, tau, k below 2^31 with a result below 2^31
 __device__ __forceinline__ u32 slot32(u32 r, u32 tau, u32 k) {
   const u64 x = static_cast<u64>(r) * tau;
@@ -436,10 +444,26 @@ __device__ __forceinline__ void scan_tile(FShared& sh, int buf, i64 t0, int wlen
   const u32 tt = static_cast<u32>(t0) + static_cast<u32>(e0);
   u32 mem[ITEMS];
 #pragma unroll
-  for (int i = 0; i < ITEMS; ++i) {
-    mem[i] = (offA + a[i]) + (tt + i) * (offB + b[i]);
-    if (e0 + i < wlen) peak = max(peak, mem[i]);
+  for (int i = 0; i < ITEMS; ++i) mem[i] = (offA + a[i]) + (tt + i) * (offB + b[i]);
+  // a tile that lies inside the phase and inside the caller's capacity needs no per-round tests
+  const bool whole = wlen == TILE && (prof_cap <= 0 || (t0 >= static_cast<i64>(first_round) && t0 + TILE <= prof_cap));
+  if (whole) {
+    u32 m = mem[0];
+#pragma unroll
+    for (int i = 1; i < ITEMS; ++i) m = max(m, mem[i]);
+    peak = max(peak, m);
+    if (prof_cap > 0) {
+      int4* dst = reinterpret_cast<int4*>(prof + t0 + e0);
+#pragma unroll
+      for (int v = 0; v < VEC; ++v)
+        dst[v] = make_int4(static_cast<int>(mem[4 * v]), static_cast<int>(mem[4 * v + 1]),
+                           static_cast<int>(mem[4 * v + 2]), static_cast<int>(mem[4 * v + 3]));
+    }
+    return;
   }
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i)
+    if (e0 + i < wlen) peak = max(peak, mem[i]);
   if (prof_cap > 0) {
     const i64 lo = first_round, hi = min_i64(t0 + wlen, prof_cap);
 #pragma unroll
@@ -503,6 +527,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
     const bool keyed = !(family == KVS_GSA && !est);          // plain GSA keeps the index order
     const bool carry = geometric && (family == KVS_GSA || est);
     const bool est_class = est && family == KVS_GBA;          // classes by the clipped estimate
+    const bool pow2 = geometric && st.alpha_num == 2 && st.alpha_den == 1 && st.beta0 <= 0;
     // arrays in schedule order (of the instance)
     const int32_t* const S_ord = (keyed ? p.sorted_s : p.s) + lo;
     const int32_t* const O_ord = (keyed ? p.sorted_o : p.o) + lo;
@@ -594,7 +619,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             if (x < nseg) {
               u32 v = static_cast<u32>(__ldg(O_ord + seg_lo + x));
               if (est_class) { const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc); v = max(v, kc); }
-              c = static_cast<u32>(class_of(sh.tau, L, v));
+              c = static_cast<u32>(pow2 ? class_pow2(Xc, v) : class_of(sh.tau, L, v));
               atomicAdd(&sh.cnt[warp][c], 1u);
             }
             if (j < 4) w0 |= c << (8 * j); else w1 |= c << (8 * (j - 4));
@@ -653,7 +678,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
         if (N > 0) len = (sim ? static_cast<i64>(ceil_div_u(N, k) - 1) * tau : static_cast<i64>(static_cast<u64>(N - 1) * tau / k)) + tau;
         sh.plen[tid] = len;
         // memory is kept modulo 2^32: the general kernel reports evaluations whose bound reaches that
-        if (walk && N > 0 && min_i64(N, static_cast<i64>(k) + 1) * (static_cast<i64>(stats.s_max) + tau) >= (static_cast<i64>(1) << 32))
+        if ((walk || event_form) && N > 0 && min_i64(N, static_cast<i64>(k) + 1) * (static_cast<i64>(stats.s_max) + tau) >= (static_cast<i64>(1) << 32))
           sh.fallback = 1;
       }
       __syncthreads();
@@ -677,31 +702,48 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
 
       // ---- per-job results ----
       if (!carry) {
-        // exactly one run per job; the rank is the position inside the class
+        // exactly one run per job; the rank is the position inside the class.  Four jobs per thread
+        // and step, loads first, so that enough memory requests are in flight.
         const u32 tau0 = sh.tau[0];
-        for (int j = seg_lo + tid; j < seg_hi; j += T) {
-          const u32 oj = static_cast<u32>(__ldg(O_JOB + j));
-          const int pos = IPERM ? __ldg(IPERM + j) : j;
-          int ph = 0;
-          bool fin = true;
-          if (geometric) ph = class_of(sh.tau, L, oj);
-          else fin = oj <= tau0;
-          const u32 rank = static_cast<u32>(pos - seg_lo - sh.ent[ph]);
-          const u32 tau = sh.tau[ph], k = sh.k[ph];
-          const u32 stt = sh.pbase[ph] + (sim ? (rank / k) * tau : slot32(rank, tau, k));
-          const u32 d = fin ? oj : tau;
-          acc.steps += d;
-          acc.hmax = max(acc.hmax, stt + d);
-          int32_t start = -1, done = -1;
-          if (fin) {
-            start = static_cast<int32_t>(stt);
-            done = static_cast<int32_t>(stt + oj);
-            acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
-          } else {
-            ++acc.unfinished;
+        constexpr int JU = 4;
+        for (int j0 = seg_lo + tid; j0 < seg_hi; j0 += JU * T) {
+          u32 oj_[JU];
+          int pos_[JU];
+#pragma unroll
+          for (int u = 0; u < JU; ++u) {
+            const int j = j0 + u * T;
+            oj_[u] = 0; pos_[u] = 0;
+            if (j < seg_hi) {
+              oj_[u] = static_cast<u32>(__ldg(O_JOB + j));
+              pos_[u] = IPERM ? __ldg(IPERM + j) : j;
+            }
           }
-          if (out_start) out_start[j] = start;
-          if (out_done) out_done[j] = done;
+#pragma unroll
+          for (int u = 0; u < JU; ++u) {
+            const int j = j0 + u * T;
+            if (j >= seg_hi) break;
+            const u32 oj = oj_[u];
+            int ph = 0;
+            bool fin = true;
+            if (geometric) ph = pow2 ? class_pow2(Xc, oj) : class_of(sh.tau, L, oj);
+            else fin = oj <= tau0;
+            const u32 rank = static_cast<u32>(pos_[u] - seg_lo - sh.ent[ph]);
+            const u32 tau = sh.tau[ph], k = sh.k[ph];
+            const u32 stt = sh.pbase[ph] + (sim ? (rank / k) * tau : slot32(rank, tau, k));
+            const u32 d = fin ? oj : tau;
+            acc.steps += d;
+            acc.hmax = max(acc.hmax, stt + d);
+            int32_t start = -1, done = -1;
+            if (fin) {
+              start = static_cast<int32_t>(stt);
+              done = static_cast<int32_t>(stt + oj);
+              acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
+            } else {
+              ++acc.unfinished;
+            }
+            if (out_start) out_start[j] = start;
+            if (out_done) out_done[j] = done;
+          }
         }
       } else {
         // The rank of a job in the phase that completes it = positions before it that leave in that
@@ -718,7 +760,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           int l = 0, f = 0;
           if (valid) {
             ov = static_cast<u32>(__ldg(O_ord + seg_lo + x));
-            if (est_class) f = class_of(sh.tau, L, min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc));
+            if (est_class) {
+              const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc);
+              f = pow2 ? class_pow2(Xc, kc) : class_of(sh.tau, L, kc);
+            }
             l = cls[x];
           }
           const u32 vm = __ballot_sync(0xffffffffu, valid);
@@ -774,14 +819,100 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
       // ---- memory profile ----
       if (event_form) {
         // SPS / SimS in exact key order with no profile wanted: the peak comes from the run ends
-        const i64* const ps = p.prefix_s + lo + st.instance + seg_lo;
-        const i64 N = nseg;
-        const i64 pr = (N + T - 1) / T;
-        const i64 i0 = min_i64(N, tid * pr), i1 = min_i64(N, i0 + pr);
-        u64 unused_flow = 0;
-        const i64 pk = sim ? sims_range_peak(O_ord + seg_lo, ps, N, sh.tau[0], sh.k[0], i0, i1, &unused_flow)
-                           : sps_range_peak(O_ord + seg_lo, ps, N, sh.tau[0], sh.k[0], i0, i1, &unused_flow);
-        acc.peak64 = max_i64(acc.peak64, pk);
+        // (see kvs_events.cuh for why the last round of every run is enough), here in 32-bit
+        // arithmetic, which the bound checked by the plan makes exact.
+        const u32* const ps32 = reinterpret_cast<const u32*>(p.prefix_s + lo + st.instance + seg_lo);   // low words
+        const u32 tau = sh.tau[0], k = sh.k[0];
+        const u32 N = static_cast<u32>(nseg);
+        const int32_t* const Ow = O_ord + seg_lo;
+        if (sim) {
+          // a batch is alone in its slot: in the last round of run i the jobs i .. end of the batch
+          // are active with progress d_i - 1
+          for (u32 i0 = tid; i0 < N; i0 += 4 * T) {
+            u32 o_[4], p_[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const u32 i = i0 + u * T;
+              o_[u] = i < N ? static_cast<u32>(__ldg(Ow + i)) : 0u;
+              p_[u] = i < N ? ps32[2 * static_cast<size_t>(i)] : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const u32 i = i0 + u * T;
+              if (i < N) {
+                const u32 bend = min(N, (i / k + 1u) * k);
+                const u32 d = min(o_[u], tau);
+                acc.peak = max(acc.peak, ps32[2 * static_cast<size_t>(bend)] - p_[u] + (bend - i) * d);
+              }
+            }
+          }
+        } else {
+          // Z[m] = sum over ranks j < m of (s_j - start_j): the jobs [i, b) active in round t hold
+          // Z[b] - Z[i] + (b - i)(t + 1) tokens.  First Z for every rank, then one candidate per run.
+          u32* const Z = reinterpret_cast<u32*>(cls);      // N + 1 words of this CTA's scratch
+          const u32 qt = tau / k, rt = tau - qt * k;
+          u32 F_run = 0;
+          for (u32 c0 = 0; c0 <= N; c0 += TILE) {
+            const u32 r = c0 + ITEMS * tid;
+            u32 q = 0, rem = 0;
+            if (r <= N) { u64 dq_, dr_; divmod_u(static_cast<u64>(r) * tau, k, &dq_, &dr_); q = static_cast<u32>(dq_); rem = static_cast<u32>(dr_); }
+            u32 f[ITEMS], tot = 0;
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) {
+              f[j] = tot;
+              if (r + j < N) tot += q;
+              rem += rt; q += qt;
+              if (rem >= k) { rem -= k; ++q; }
+            }
+            u32 incl = tot;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+              const u32 y = __shfl_up_sync(0xffffffffu, incl, d);
+              if (lane >= d) incl += y;
+            }
+            __syncthreads();
+            if (lane == 31) sh.redA[warp] = incl;
+            __syncthreads();
+            const u32 w = lane < WARPS ? sh.redA[lane] : 0u;
+            u32 wi = w;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+              const u32 y = __shfl_up_sync(0xffffffffu, wi, d);
+              if (lane >= d) wi += y;
+            }
+            const u32 off = F_run + __shfl_sync(0xffffffffu, wi - w, warp) + (incl - tot);
+            F_run += __shfl_sync(0xffffffffu, wi, 31);
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j)
+              if (r + j <= N) Z[r + j] = ps32[2 * static_cast<size_t>(r + j)] - (off + f[j]);
+          }
+          __syncthreads();
+          for (u32 c0 = 0; c0 < N; c0 += TILE) {
+            const u32 r = c0 + ITEMS * tid;
+            if (r >= N) continue;
+            u64 dq_, dr_;
+            divmod_u(static_cast<u64>(r) * tau, k, &dq_, &dr_);
+            u32 q = static_cast<u32>(dq_), rem = static_cast<u32>(dr_);
+            u32 o_[ITEMS], z_[ITEMS];
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) {
+              o_[j] = r + j < N ? static_cast<u32>(__ldg(Ow + r + j)) : 0u;
+              z_[j] = r + j < N ? Z[r + j] : 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) {
+              if (r + j < N) {
+                const u32 t1 = q + min(o_[j], tau);                       // last round of the run, plus one
+                const u64 x = static_cast<u64>(t1) * k + (tau - 1u);      // b = ranks that start before t1
+                const u32 b = (x >> 32) ? static_cast<u32>(min(static_cast<u64>(N), x / tau)) : min(N, static_cast<u32>(x) / tau);
+                acc.peak = max(acc.peak, Z[b] - z_[j] + (b - (r + j)) * t1);
+              }
+              rem += rt; q += qt;
+              if (rem >= k) { rem -= k; ++q; }
+            }
+          }
+          __syncthreads();     // Z is scratch of the next window too
+        }
       } else if (walk) {
         for (int ph = 0; ph < L; ++ph) {
           const int N = static_cast<int>(sh.np[ph]);
