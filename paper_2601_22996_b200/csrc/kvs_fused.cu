@@ -36,13 +36,20 @@ constexpr int WARPS = T / 32;
 constexpr int VEC = ITEMS / 4;
 constexpr int RPT = 4;                       // consecutive ranks per thread in the run visit
 constexpr int MAXP = KVS_MAX_PHASES;
+constexpr int RINGW = 2 * TILE + (2 * TILE) / 8;
+constexpr int GCOL = 2049;
+static_assert((TILE & (TILE - 1)) == 0 && ITEMS % 4 == 0 && ITEMS <= 32 && 32 % ITEMS == 0, "tile layout");
 constexpr u32 TIME_LIMIT = 0x7fffffffu - 4u * TILE;   // phase ends stay below this
 
 typedef unsigned __int128 u128;
 
 struct FShared {
-  uint4 dA[2][TILE / 4];      // two-tile ring: difference arrays of the constant terms
-  uint4 dB[2][TILE / 4];      //                and of the slopes
+  // two-tile ring of difference arrays: constant terms and slopes.  Round e of the ring (0 <= e <
+  // 2*TILE) lives at word e + 4*(e/32): four spare words after every 32 keep the 16-byte loads of
+  // the scan (a thread owns ITEMS consecutive rounds) free of bank conflicts while the index of an
+  // event stays a shift and an add.
+  u32 dA[RINGW];
+  u32 dB[RINGW];
   u128 pw_a[MAXP + 1];
   u128 pw_b[MAXP + 1];
   u64 taupre[MAXP + 1];       // sum of tau_q over q < p
@@ -53,6 +60,7 @@ struct FShared {
   i64 n_runs;
   u32 tau[MAXP], k[MAXP], pbase[MAXP], np[MAXP];
   u32 cnt[WARPS][MAXP];       // per-warp class counts, then ranks before each warp's segment
+  u32 gcol[GCOL];             // the current phase's column of the rank table (windows of up to (GCOL-1)*256 jobs)
   u32 redA[32], redB[32];
   int red32[32];
   int ent[MAXP + 1];          // class boundaries in key order
@@ -142,11 +150,11 @@ __device__ __forceinline__ u32 slot32(u32 r, u32 tau, u32 k) {
   return static_cast<u32>(x / k);
 }
 
-// Word of round e of a tile: thread t owns rounds ITEMS*t .. ITEMS*t+ITEMS-1 as VEC 4-word vectors,
-// vector c of thread t at vector index c*T + t, so that a warp's vector access is contiguous.
-__device__ __forceinline__ int slot(int e) { return ((((e >> 2) % VEC) * T + e / ITEMS) << 2) + (e & 3); }
 // Word of the round `rel` rounds after the origin of ring half `buf`, 0 <= rel < 2*TILE.
-__device__ __forceinline__ int ring(int buf, int rel) { return ((buf ^ (rel >= TILE ? 1 : 0)) * TILE) + slot(rel & (TILE - 1)); }
+__device__ __forceinline__ int ring(int buf, int rel) {
+  const int e = (buf * TILE + rel) & (2 * TILE - 1);
+  return e + ((e >> 5) << 2);
+}
 
 // One phase as the run visit sees it.  Positions are relative to the window, in schedule order.
 // Exact keys: the participants are the positions [x_lo, x_hi) and the rank is the offset from x_lo.
@@ -158,6 +166,7 @@ struct PhaseView {
   const int32_t* O;
   const unsigned char* cls;
   const u32* G;
+  const u32* gcol;        // column ph of G in shared memory, or NULL
   int L, ph, nsegs;
   int x_lo, x_hi;
   u32 tau, k, qt, rt;     // tau = qt*k + rt
@@ -166,6 +175,11 @@ struct PhaseView {
 };
 
 constexpr int SEG = 256;  // positions per warp step: 8 consecutive positions per lane
+
+// participants of the phase before segment `seg`
+__device__ __forceinline__ int rank_before(const PhaseView& P, int seg) {
+  return static_cast<int>(P.gcol ? P.gcol[seg] : P.G[seg * P.L + P.ph]);
+}
 
 // The 8 positions of one lane in segment `seg`: bit j of `bits` is set if position xb + j takes part,
 // and those positions have the consecutive ranks r_first, r_first + 1, ...
@@ -194,7 +208,7 @@ __device__ __forceinline__ LaneGroup lane_group(const PhaseView& P, int seg) {
       const int y = __shfl_up_sync(0xffffffffu, incl, d);
       if (lane >= d) incl += y;
     }
-    g.r_first = static_cast<int>(P.G[seg * P.L + P.ph]) + incl - cnt;
+    g.r_first = rank_before(P, seg) + incl - cnt;
   } else {
     g.r_first = seg * SEG + 8 * lane;
     g.xb = P.x_lo + g.r_first;
@@ -210,10 +224,10 @@ __device__ __forceinline__ void segment_range(const PhaseView& P, int ra, int rb
   if (FILTER) {
     // G[.][ph] is nondecreasing over the nsegs + 1 rows; last row = number of participants
     int a = 0, b = P.nsegs;               // largest seg with G[seg] <= ra
-    while (a < b) { const int m = (a + b + 1) >> 1; if (static_cast<int>(P.G[m * P.L + P.ph]) <= ra) a = m; else b = m - 1; }
+    while (a < b) { const int m = (a + b + 1) >> 1; if (rank_before(P, m) <= ra) a = m; else b = m - 1; }
     *seg_a = a;
     a = 0; b = P.nsegs;                   // smallest seg with G[seg] >= rb
-    while (a < b) { const int m = (a + b) >> 1; if (static_cast<int>(P.G[m * P.L + P.ph]) >= rb) b = m; else a = m + 1; }
+    while (a < b) { const int m = (a + b) >> 1; if (rank_before(P, m) >= rb) b = m; else a = m + 1; }
     *seg_b = a;
   } else {
     *seg_a = ra / SEG;
@@ -229,8 +243,8 @@ template <bool SIM, bool FILTER>
 __device__ __forceinline__ void visit_runs(FShared& sh, const PhaseView& P, int ra, int rb, int trel, int buf,
                                            bool dense, bool combine) {
   if (ra >= rb) return;
-  u32* const dA = reinterpret_cast<u32*>(sh.dA);
-  u32* const dB = reinterpret_cast<u32*>(sh.dB);
+  u32* const dA = sh.dA;
+  u32* const dB = sh.dB;
   const u32 tau = P.tau, k = P.k;
   const int warp = threadIdx.x >> 5;
   int seg_a, seg_b;
@@ -365,8 +379,8 @@ __device__ __forceinline__ void insert_far_ends(FShared& sh, const PhaseView& P,
   if (r_hi > N) r_hi = N;
   if (r_lo >= r_hi) return;
   const int ra = static_cast<int>(r_lo), rb = static_cast<int>(r_hi);
-  u32* const dA = reinterpret_cast<u32*>(sh.dA);
-  u32* const dB = reinterpret_cast<u32*>(sh.dB);
+  u32* const dA = sh.dA;
+  u32* const dB = sh.dB;
   const int warp = threadIdx.x >> 5;
   int seg_a, seg_b;
   segment_range<FILTER>(P, ra, rb, &seg_a, &seg_b);
@@ -384,7 +398,7 @@ __device__ __forceinline__ void insert_far_ends(FShared& sh, const PhaseView& P,
       const int ts = a0 + ((static_cast<int>(q) - a0) / TILE) * TILE;   // origin of the tile the run started in
       if (static_cast<int>(end) >= ts + 2 * TILE && static_cast<int>(end) >= u0 && static_cast<int>(end) < u0 + wlen && end < P.len) {
         const u32 c = si + 1u - P.base - q;
-        const int ei = buf * TILE + slot(static_cast<int>(end) - u0);
+        const int ei = ring(buf, static_cast<int>(end) - u0);
         atomicAdd(&dA[ei], 0u - c);
         atomicAdd(&dB[ei], 0xffffffffu);
       }
@@ -410,11 +424,14 @@ __device__ __forceinline__ void scan_tile(FShared& sh, int buf, i64 t0, int wlen
   const int tid = threadIdx.x;
   const uint4 zero = make_uint4(0, 0, 0, 0);
   u32 a[ITEMS], b[ITEMS];
+  const int w0 = ring(buf, ITEMS * tid);       // the thread's ITEMS rounds are consecutive words
 #pragma unroll
   for (int v = 0; v < VEC; ++v) {
-    const uint4 x = sh.dA[buf][v * T + tid], y = sh.dB[buf][v * T + tid];
-    sh.dA[buf][v * T + tid] = zero;
-    sh.dB[buf][v * T + tid] = zero;
+    uint4* const pa = reinterpret_cast<uint4*>(&sh.dA[w0 + 4 * v]);
+    uint4* const pb = reinterpret_cast<uint4*>(&sh.dB[w0 + 4 * v]);
+    const uint4 x = *pa, y = *pb;
+    *pa = zero;
+    *pb = zero;
     a[4 * v] = x.x; a[4 * v + 1] = x.y; a[4 * v + 2] = x.z; a[4 * v + 3] = x.w;
     b[4 * v] = y.x; b[4 * v + 1] = y.y; b[4 * v + 2] = y.z; b[4 * v + 3] = y.w;
   }
@@ -499,8 +516,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
   u32* const G = reinterpret_cast<u32*>(cls + ((p.max_jobs + SEG + 15) & ~static_cast<i64>(15)));
   u32* const fin_start = reinterpret_cast<u32*>(p.fin_rank) + static_cast<i64>(blockIdx.x) * p.max_jobs;
   {
-    const uint4 zero = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < 2 * (TILE / 4); i += T) { (&sh.dA[0][0])[i] = zero; (&sh.dB[0][0])[i] = zero; }
+    for (int i = tid; i < RINGW; i += T) { sh.dA[i] = 0; sh.dB[i] = 0; }
   }
 
   for (;;) {
@@ -920,6 +936,12 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           PhaseView P;
           P.S = S_ord + seg_lo; P.O = O_ord + seg_lo;
           P.cls = cls; P.G = G; P.L = L; P.ph = ph; P.nsegs = nsegs;
+          P.gcol = nullptr;
+          if (carry && nsegs < GCOL) {
+            for (int seg = tid; seg <= nsegs; seg += T) sh.gcol[seg] = G[seg * L + ph];
+            P.gcol = sh.gcol;
+            __syncthreads();
+          }
           P.x_lo = carry ? 0 : sh.ent[ph];
           P.x_hi = sh.ent[ph + 1];
           P.tau = sh.tau[ph]; P.k = sh.k[ph];
