@@ -168,6 +168,7 @@ struct PhaseView {
   const u32* G;
   const u32* gcol;        // column ph of G in shared memory, or NULL
   int L, ph, nsegs;
+  int n_src;              // positions of the window (S and O may be read below this index)
   int x_lo, x_hi;
   u32 tau, k, qt, rt;     // tau = qt*k + rt
   u32 len;                // rounds of the phase
@@ -183,7 +184,15 @@ __device__ __forceinline__ int rank_before(const PhaseView& P, int seg) {
 
 // The 8 positions of one lane in segment `seg`: bit j of `bits` is set if position xb + j takes part,
 // and those positions have the consecutive ranks r_first, r_first + 1, ...
-struct LaneGroup { u32 bits; int r_first; int xb; };
+// With FILTER, `fbits` marks the participants whose leaving class is this phase (they complete here;
+// the others are killed at the end of their slot and their response length is not needed).
+struct LaneGroup { u32 bits; u32 fbits; int r_first; int xb; };
+
+// Bit j of the result is set iff byte j of `w` is >= (ge) or == the byte replicated in `p4`.
+__device__ __forceinline__ u32 byte_mask4(u32 w, u32 p4, bool ge) {
+  const u32 m = (ge ? __vcmpgeu4(w, p4) : __vcmpeq4(w, p4)) & 0x08040201u;
+  return (m | (m >> 8) | (m >> 16) | (m >> 24)) & 15u;
+}
 
 template <bool FILTER>
 __device__ __forceinline__ LaneGroup lane_group(const PhaseView& P, int seg) {
@@ -194,13 +203,9 @@ __device__ __forceinline__ LaneGroup lane_group(const PhaseView& P, int seg) {
     const uint2 cw = *reinterpret_cast<const uint2*>(P.cls + g.xb);
     const int room = P.x_hi - g.xb;                        // positions of this lane below x_hi
     const u32 lim = room >= 8 ? 0xffu : (room > 0 ? (1u << room) - 1u : 0u);
-    u32 bits = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const u32 c = ((j < 4 ? cw.x : cw.y) >> (8 * (j & 3))) & 255u;
-      if (c >= static_cast<u32>(P.ph)) bits |= 1u << j;
-    }
-    g.bits = bits & lim;
+    const u32 p4 = static_cast<u32>(P.ph) * 0x01010101u;
+    g.bits = (byte_mask4(cw.x, p4, true) | byte_mask4(cw.y, p4, true) << 4) & lim;
+    g.fbits = (byte_mask4(cw.x, p4, false) | byte_mask4(cw.y, p4, false) << 4) & lim;
     int incl = __popc(g.bits);
     const int cnt = incl;
 #pragma unroll
@@ -214,6 +219,7 @@ __device__ __forceinline__ LaneGroup lane_group(const PhaseView& P, int seg) {
     g.xb = P.x_lo + g.r_first;
     const int room = P.x_hi - g.xb;
     g.bits = room >= 8 ? 0xffu : (room > 0 ? (1u << room) - 1u : 0u);
+    g.fbits = g.bits;
   }
   return g;
 }
@@ -247,9 +253,21 @@ __device__ __forceinline__ void visit_runs(FShared& sh, const PhaseView& P, int 
   u32* const dB = sh.dB;
   const u32 tau = P.tau, k = P.k;
   const int warp = threadIdx.x >> 5;
+  // 16-byte loads need aligned rows; without the filter a lane's first position is x_lo + 8*(...)
+  const bool vec = ((reinterpret_cast<uintptr_t>(P.S) | reinterpret_cast<uintptr_t>(P.O)) & 15u) == 0 && (FILTER || (P.x_lo & 3) == 0);
   int seg_a, seg_b;
   segment_range<FILTER>(P, ra, rb, &seg_a, &seg_b);
   for (int seg = seg_a + warp; seg < seg_b; seg += WARPS) {
+    // The prompt lengths of the lane's eight positions do not depend on which of them take part:
+    // where all eight exist and the rows are 16-byte aligned they are requested first, as two
+    // 16-byte loads, so that they travel together with the class bytes instead of after them.
+    const int xb0 = (FILTER ? 0 : P.x_lo) + seg * SEG + 8 * static_cast<int>(lane_id());
+    const bool vload = vec && xb0 + 8 <= P.n_src;
+    uint4 a0 = make_uint4(0, 0, 0, 0), a1 = a0;
+    if (vload) {
+      a0 = __ldg(reinterpret_cast<const uint4*>(P.S + xb0));
+      a1 = __ldg(reinterpret_cast<const uint4*>(P.S + xb0) + 1);
+    }
     const LaneGroup g = lane_group<FILTER>(P, seg);
     // of this lane's participants, entries [skip, skip + take) have ranks inside [ra, rb)
     const int cnt = __popc(g.bits);
@@ -257,12 +275,24 @@ __device__ __forceinline__ void visit_runs(FShared& sh, const PhaseView& P, int 
     const int take = min(cnt, rb - g.r_first) - skip;
     if (__ballot_sync(0xffffffffu, take > 0) == 0) continue;
     u32 s_[8], o_[8];
+    // a killed run lasts tau rounds whatever its response length: only completing jobs load it
+    const u32 need_o = take > 0 ? g.fbits : 0u;
+    if (vload) {
+      s_[0] = a0.x; s_[1] = a0.y; s_[2] = a0.z; s_[3] = a0.w; s_[4] = a1.x; s_[5] = a1.y; s_[6] = a1.z; s_[7] = a1.w;
+      if (FILTER) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      s_[j] = 0; o_[j] = 0;
-      if (take > 0 && (g.bits >> j & 1u)) {
-        s_[j] = static_cast<u32>(__ldg(P.S + g.xb + j));
-        o_[j] = static_cast<u32>(__ldg(P.O + g.xb + j));
+        for (int j = 0; j < 8; ++j) o_[j] = (need_o >> j & 1u) ? static_cast<u32>(__ldg(P.O + g.xb + j)) : 0xffffffffu;
+      } else {
+        const uint4 b0 = take > 0 ? __ldg(reinterpret_cast<const uint4*>(P.O + g.xb)) : make_uint4(0, 0, 0, 0);
+        const uint4 b1 = take > 0 ? __ldg(reinterpret_cast<const uint4*>(P.O + g.xb) + 1) : make_uint4(0, 0, 0, 0);
+        o_[0] = b0.x; o_[1] = b0.y; o_[2] = b0.z; o_[3] = b0.w; o_[4] = b1.x; o_[5] = b1.y; o_[6] = b1.z; o_[7] = b1.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        s_[j] = 0; o_[j] = 0xffffffffu;
+        if (take > 0 && (g.bits >> j & 1u)) s_[j] = static_cast<u32>(__ldg(P.S + g.xb + j));
+        if (need_o >> j & 1u) o_[j] = static_cast<u32>(__ldg(P.O + g.xb + j));
       }
     }
     u32 q = 0, rem = 0;      // start offset of the current rank inside the phase and its remainder
@@ -942,6 +972,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             P.gcol = sh.gcol;
             __syncthreads();
           }
+          P.n_src = nseg;
           P.x_lo = carry ? 0 : sh.ent[ph];
           P.x_hi = sh.ent[ph + 1];
           P.tau = sh.tau[ph]; P.k = sh.k[ph];
