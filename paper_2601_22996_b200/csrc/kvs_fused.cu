@@ -395,6 +395,168 @@ __device__ __forceinline__ void visit_runs(FShared& sh, const PhaseView& P, int 
   }
 }
 
+// Exclusive block scan of a small per-thread count; returns this thread's offset, total in *total.
+__device__ __forceinline__ int block_count_scan(int v, int* red32, int* total) {
+  int incl = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, d);
+    if (static_cast<int>(lane_id()) >= d) incl += y;
+  }
+  const int warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane_id() == 31) red32[warp] = incl;
+  __syncthreads();
+  const int w = (lane_id() < WARPS) ? red32[lane_id()] : 0;
+  int wi = w;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, wi, d);
+    if (static_cast<int>(lane_id()) >= d) wi += y;
+  }
+  *total = __shfl_sync(0xffffffffu, wi, 31);
+  return __shfl_sync(0xffffffffu, wi - w, warp) + (incl - v);
+}
+
+// Participants of a phase as a list (used once fewer than half of a window's positions still take
+// part): rank r < C is the (s, o) pair cur[r], rank r >= C is position src + (r - C) of the
+// window (jobs that enter in this phase).
+struct ListView {
+  const uint2* cur;
+  int C;
+  int src;
+};
+
+// Run visit over a list: ranks [ra, rb), one to four consecutive ranks per thread, so that a tile
+// with few runs is spread over the whole block instead of a few warps.  Adds the two events of
+// every run and appends the killed jobs to `nxt`; returns the new length of `nxt`.  Block-wide
+// (two barriers per 2048 ranks for the positions of the survivors).
+__device__ __forceinline__ int visit_list(FShared& sh, const PhaseView& P, const ListView& V, uint2* nxt, int C_next,
+                                          int ra, int rb, int trel, int buf, bool dense) {
+  const int tid = threadIdx.x, lane = lane_id();
+  u32* const dA = sh.dA;
+  u32* const dB = sh.dB;
+  const u32 tau = P.tau, k = P.k;
+  for (int c0 = ra; c0 < rb;) {
+    const int left = rb - c0;
+    const int rpt = left > 2 * T ? RPT : (left > T ? 2 : 1);
+    const int r_first = c0 + tid * rpt;
+    c0 += T * rpt;
+    uint2 keep[RPT];
+    u32 cmask = 0;
+    if (r_first - lane * rpt < rb) {   // warps past the end of the range skip the visit
+      u32 s_[RPT], o_[RPT];
+      bool on[RPT];
+#pragma unroll
+      for (int j = 0; j < RPT; ++j) {
+        const int r = r_first + j;
+        on[j] = j < rpt && r < rb;
+        s_[j] = 0; o_[j] = 0;
+        if (on[j]) {
+          if (r < V.C) { const uint2 e = V.cur[r]; s_[j] = e.x; o_[j] = e.y; }
+          else { s_[j] = static_cast<u32>(__ldg(P.S + V.src + (r - V.C))); o_[j] = static_cast<u32>(__ldg(P.O + V.src + (r - V.C))); }
+        }
+      }
+      u32 q = 0, rem = 0;
+      if (on[0]) {
+        u64 dq_, dr_;
+        divmod_u(static_cast<u64>(r_first) * tau, k, &dq_, &dr_);
+        q = static_cast<u32>(dq_);
+        rem = static_cast<u32>(dr_);
+      }
+      int seg_key = 0x7fffffff;
+      u32 seg_all = 0, seg_full = 0, seg_cnt = 0;
+#pragma unroll
+      for (int j = 0; j < RPT; ++j) {
+        if (on[j]) {
+          const u32 oi = o_[j];
+          const u32 d = oi < tau ? oi : tau;
+          if (oi > tau) { keep[j] = make_uint2(s_[j], oi); cmask |= 1u << j; }
+          const u32 c = s_[j] + 1u - P.base - q;
+          const int srel = static_cast<int>(q) - trel;
+          int sidx = ring(buf, srel), eidx = -1;
+          if (q + d < P.len) {
+            const u32 erel = static_cast<u32>(srel) + d;
+            if (erel < 2u * TILE) eidx = ring(buf, static_cast<int>(erel));
+          }
+          if (dense) {
+            if (seg_key == 0x7fffffff) seg_key = srel;
+            if (srel == seg_key) {
+              seg_all += c; seg_cnt += 1u;
+              sidx = -1;
+              if (d == tau) { seg_full += c; seg_cnt += 1u << 16; eidx = -1; }
+            }
+          }
+          if (sidx >= 0) { atomicAdd(&dA[sidx], c); atomicAdd(&dB[sidx], 1u); }
+          if (eidx >= 0) { atomicAdd(&dA[eidx], 0u - c); atomicAdd(&dB[eidx], 0xffffffffu); }
+          rem += P.rt; q += P.qt;
+          if (rem >= k) { rem -= k; ++q; }
+        }
+      }
+      if (dense) {
+        const u32 has = __ballot_sync(0xffffffffu, seg_key != 0x7fffffff);
+        const u32 before = has & lanemask_lt();
+        const int src = (seg_key == 0x7fffffff && before) ? 31 - __clz(before) : lane;
+        const int key = __shfl_sync(0xffffffffu, seg_key, src);
+        u32 va = seg_all, vf = seg_full, vn = seg_cnt;
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+          const int kk = __shfl_up_sync(0xffffffffu, key, dd);
+          const u32 ya = __shfl_up_sync(0xffffffffu, va, dd), yf = __shfl_up_sync(0xffffffffu, vf, dd);
+          const u32 yn = __shfl_up_sync(0xffffffffu, vn, dd);
+          if (lane >= dd && kk == key) { va += ya; vf += yf; vn += yn; }
+        }
+        const int next_key = __shfl_down_sync(0xffffffffu, key, 1);
+        if (key != 0x7fffffff && (lane == 31 || next_key != key)) {
+          const int si = ring(buf, key);
+          atomicAdd(&dA[si], va);
+          atomicAdd(&dB[si], vn & 0xffffu);
+          const u32 n_full = vn >> 16;
+          if (n_full && static_cast<u32>(key + trel) + tau < P.len) {
+            const int ei = ring(buf, key + static_cast<int>(tau));
+            atomicAdd(&dA[ei], 0u - vf);
+            atomicAdd(&dB[ei], 0u - n_full);
+          }
+        }
+      }
+    }
+    int total;
+    int off = C_next + block_count_scan(__popc(cmask), sh.red32, &total);
+#pragma unroll
+    for (int j = 0; j < RPT; ++j)
+      if (cmask >> j & 1u) nxt[off++] = keep[j];
+    C_next += total;
+  }
+  return C_next;
+}
+
+// insert_far_ends for a list: slices longer than a tile only.
+__device__ __forceinline__ void insert_far_ends_list(FShared& sh, const PhaseView& P, const ListView& V, int N, int a0,
+                                                     int u0, int wlen, int buf) {
+  if (u0 <= TILE) return;
+  const u32 lo = static_cast<u32>(u0) > P.tau ? static_cast<u32>(u0) - P.tau : 0u, hi = static_cast<u32>(u0 - TILE);
+  i64 r_lo = ceil_div_u(static_cast<u64>(lo) * P.k, P.tau), r_hi = ceil_div_u(static_cast<u64>(hi) * P.k, P.tau);
+  if (r_hi > N) r_hi = N;
+  for (i64 r0 = r_lo; r0 < r_hi; r0 += T) {
+    const i64 rr = r0 + threadIdx.x;
+    if (rr < r_hi) {
+      const int r = static_cast<int>(rr);
+      u32 si, oi;
+      if (r < V.C) { const uint2 e = V.cur[r]; si = e.x; oi = e.y; }
+      else { si = static_cast<u32>(__ldg(P.S + V.src + (r - V.C))); oi = static_cast<u32>(__ldg(P.O + V.src + (r - V.C))); }
+      const u32 q = slot32(static_cast<u32>(r), P.tau, P.k);
+      const u32 end = q + (oi < P.tau ? oi : P.tau);
+      const int ts = a0 + ((static_cast<int>(q) - a0) / TILE) * TILE;
+      if (static_cast<int>(end) >= ts + 2 * TILE && static_cast<int>(end) >= u0 && static_cast<int>(end) < u0 + wlen && end < P.len) {
+        const u32 c = si + 1u - P.base - q;
+        const int ei = ring(buf, static_cast<int>(end) - u0);
+        atomicAdd(&sh.dA[ei], 0u - c);
+        atomicAdd(&sh.dB[ei], 0xffffffffu);
+      }
+    }
+  }
+}
+
 // Slices longer than a tile: ends that land two or more tiles after the run's start were not
 // inserted when the run was visited; pick them up when their tile comes.  u0 = offset of this
 // tile's origin inside the phase, a0 = the same for the phase's first tile (0 or slightly negative).
@@ -544,6 +706,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
   // per-CTA scratch: class bytes of the current window (padded to whole segments), then the rank table
   unsigned char* const cls = reinterpret_cast<unsigned char*>(p.lists) + static_cast<i64>(blockIdx.x) * KVS_CTA_SCRATCH(p.max_jobs);
   u32* const G = reinterpret_cast<u32*>(cls + ((p.max_jobs + SEG + 15) & ~static_cast<i64>(15)));
+  // two lists of (s, o) pairs for windows of which fewer than half of the positions still take part
+  uint2* const list0 = reinterpret_cast<uint2*>(reinterpret_cast<unsigned char*>(G) + ((static_cast<size_t>(p.max_jobs) / SEG + 2) * MAXP * 4));
+  uint2* const list1 = list0 + (p.max_jobs + 1);
   u32* const fin_start = reinterpret_cast<u32*>(p.fin_rank) + static_cast<i64>(blockIdx.x) * p.max_jobs;
   {
     for (int i = tid; i < RINGW; i += T) { sh.dA[i] = 0; sh.dB[i] = 0; }
@@ -960,6 +1125,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           __syncthreads();     // Z is scratch of the next window too
         }
       } else if (walk) {
+        bool list_mode = false;
+        uint2* cur = list0;
+        uint2* nxt = list1;
+        int C = 0;
         for (int ph = 0; ph < L; ++ph) {
           const int N = static_cast<int>(sh.np[ph]);
           if (N == 0) continue;
@@ -981,6 +1150,22 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           P.base = sh.pbase[ph];
           const bool combine = sim && P.k >= 32;
           const bool dense = !sim && P.tau < TILE && P.k >= 4 * P.tau;
+          ListView V;
+          V.cur = cur; V.C = C; V.src = sh.ent[ph];
+          if (carry && !list_mode && 2 * N <= nseg) {
+            // from here on the participants are kept as a list in rank order: first this phase's
+            for (int seg = warp; seg < nsegs; seg += WARPS) {
+              const LaneGroup g = lane_group<true>(P, seg);
+              int r = g.r_first;
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                if (g.bits >> j & 1u) cur[r++] = make_uint2(static_cast<u32>(__ldg(P.S + g.xb + j)), static_cast<u32>(__ldg(P.O + g.xb + j)));
+            }
+            list_mode = true;
+            V.C = N;
+            __syncthreads();
+          }
+          int C_next = 0;
           // idle rounds before this phase (window release) hold nothing
           if (prof_cap > 0)
             for (i64 t = written_to + tid; t < P.base && t < prof_cap; t += T) prof[t] = 0;
@@ -1005,11 +1190,13 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             cq += dq; cr += dr;
             if (cr >= utau) { cr -= utau; ++cq; }
             if (sim) visit_runs<true, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
+            else if (list_mode) C_next = visit_list(sh, P, V, nxt, C_next, r_next, r_b, u0, buf, dense);
             else if (carry) visit_runs<false, true>(sh, P, r_next, r_b, u0, buf, dense, combine);
             else visit_runs<false, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             r_next = r_b;
             if (P.tau > TILE) {
-              if (carry) insert_far_ends<true>(sh, P, sim, N, a0, u0, wlen, buf);
+              if (list_mode) insert_far_ends_list(sh, P, V, N, a0, u0, wlen, buf);
+              else if (carry) insert_far_ends<true>(sh, P, sim, N, a0, u0, wlen, buf);
               else insert_far_ends<false>(sh, P, sim, N, a0, u0, wlen, buf);
             }
             __syncthreads();
@@ -1017,6 +1204,11 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             buf ^= 1;
           }
           written_to = static_cast<i64>(P.base) + P.len;
+          if (list_mode) {
+            __syncthreads();               // the list of killed jobs is complete before it is read
+            uint2* const tmp = cur; cur = nxt; nxt = tmp;
+            C = C_next;
+          }
         }
       }
       base = sh.base_next;

@@ -23,9 +23,11 @@ constexpr int KVS_EVAL_ITEMS = KVS_EVAL_ITEMS_CFG;        // rounds per thread a
 constexpr int KVS_EVAL_MIN_CTAS = KVS_EVAL_MIN_CTAS_CFG;  // CTAs per SM the register allocation aims at
 constexpr int KVS_TILE = KVS_EVAL_THREADS * KVS_EVAL_ITEMS;  // rounds per shared-memory tile
 
-// Scratch bytes of one CTA of the fused kernels (carry lists of the general kernel; class bytes and
-// rank table of the fast kernel), for instances of at most max_jobs jobs.
-#define KVS_CTA_SCRATCH(max_jobs) (16 * static_cast<i64>(max_jobs) + 2048)
+// Scratch bytes of one CTA of the fused kernels (carry lists of the general kernel; class bytes, rank
+// table - about 2.5 bytes per job - and two lists of (s, o) pairs of the fast kernel), for instances
+// of at most max_jobs jobs.
+// A multiple of 256 bytes, so that every CTA's block keeps the 16-byte alignment its vector accesses need.
+#define KVS_CTA_SCRATCH(max_jobs) ((20 * static_cast<i64>(max_jobs) + 4096 + 255) & ~static_cast<i64>(255))
 
 // Per-instance statistics produced by the first kernel.
 struct InstStats {
