@@ -25,6 +25,11 @@ sys.path.insert(0, ROOT)
 from paper_2601_22996_b200 import workloads  # noqa: E402
 
 METRIC, UNIT = "schedule_evaluation_job_steps_per_sec", "job-steps/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_fused_eval launch, from the ncu capture summarised in
+# profiles/k_fused_eval_c5.md (592 instances of config 5, all four families: 2,368 evaluations, 4.727 GB).
+# Traffic grows with the number of evaluations (each CTA works on one at a time), so a launch is scaled
+# by its evaluation count.  Valid for the kernel state named in that file; set to None when the kernel changes.
+C5_TRAFFIC_BYTES_PER_EVALUATION = 4.726584e9 / 2368
 WORKLOADS = {
     # name: (generator, instances, jobs per instance, families, description)
     "c2": ("config2", 1024, 10_000, ["GBA", "GSA"], "config 2: 1,024 instances x 10,000 jobs, M in {2^17..2^24}, GBA+GSA"),
@@ -284,6 +289,9 @@ def run_ours(args):
     alg_bytes = 8 * N + 8 * P * n + 4 * rounds + 57 * P
     peak_gbs, peak_kind = load_peaks()
     achieved = alg_bytes / (build_avg * 1e-3) / 1e9
+    traffic = None
+    if name == "c5" and len(fams) == 4 and C5_TRAFFIC_BYTES_PER_EVALUATION:
+        traffic = C5_TRAFFIC_BYTES_PER_EVALUATION * P
     line = {
         "metric": METRIC, "value": steps_all / sec_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * sec_per_step, "higher_is_better": True, "scaling": "weak",
@@ -294,7 +302,7 @@ def run_ours(args):
         "evaluations_per_sec": evals_all / sec_per_step,
         "kernels_ms": {"k_stats_sort": sort_avg, "k_fused_eval+k_build_eval": build_avg},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
-                     "traffic": None, "peak_kind": peak_kind, "kernel": "k_fused_eval", "algorithmic_bytes": alg_bytes},
+                     "traffic": traffic, "peak_kind": peak_kind, "kernel": "k_fused_eval", "algorithmic_bytes": alg_bytes},
         "gpu_launches": 3 * args.steps, "clocks": clocks,
     }
     if e2e:
