@@ -102,18 +102,19 @@ def test_config2_full_size_sampled(par):
     _check_sample(par, inst, settings, window, n, out, ev, sorted(rng.choice(settings.shape[0], 24, replace=False)))
 
 
-def test_config5_large_subset_sampled(par):
-    inst, settings, window, n, out, ev, _ = _bench_call(par, "c5", 2048)
+def test_config5_full_size_sampled(par):
+    """The whole stress config (16,384 instances, 65,536 evaluations) in one call, as bench.py times it."""
+    inst, settings, window, n, out, ev, _ = _bench_call(par, "c5", 16384)
     _check_properties(settings, n, out, ev, inst)
     rng = np.random.default_rng(5)
     _check_sample(par, inst, settings, window, n, out, ev, sorted(rng.choice(settings.shape[0], 24, replace=False)))
 
 
 def test_config3_online_sampled(par):
-    inst, settings, window, n, out, ev, _ = _bench_call(par, "c3", 64)
+    inst, settings, window, n, out, ev, _ = _bench_call(par, "c3", 256)
     assert int((ev["status"] != 0).sum()) == 0 and int(ev["n_unfinished"].sum()) == 0
     rng = np.random.default_rng(3)
-    _check_sample(par, inst, settings, window, n, out, ev, sorted(rng.choice(settings.shape[0], 6, replace=False)))
+    _check_sample(par, inst, settings, window, n, out, ev, sorted(rng.choice(settings.shape[0], 8, replace=False)))
 
 
 def test_config4_sweep_full_size_sampled(par):
