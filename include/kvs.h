@@ -170,8 +170,11 @@ int kvs_evaluate_built(kvs_ctx* ctx, const kvs_instances* inst, const kvs_settin
 /* Same as kvs_evaluate_built for HOST inputs and HOST scalar results: copies job_off, s, o
  * (and o_est, arrival) to the workspace, runs the fused path, and copies the per-evaluation
  * scalars back.  Every pointer of `inst` and of `ev` is a HOST pointer here (pinned memory
- * makes the copies asynchronous); `ev->profile` must be NULL.  The call returns after the
- * stream has been synchronised. */
+ * makes the copies asynchronous); `ev->profile` must be NULL.  The instances are worked off in up
+ * to 16 chunks: the jobs of the next chunk are copied on a second stream while the kernels of the
+ * current one run, so the settings may come in any order but are evaluated grouped by instance
+ * (results are returned in the caller's order).  job_off is read on the host and must be
+ * nondecreasing.  The call returns after the stream has been synchronised. */
 int kvs_evaluate_built_host(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings,
                             int64_t P, const kvs_eval_out* ev);
 

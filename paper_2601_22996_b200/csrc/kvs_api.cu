@@ -1,11 +1,15 @@
 // C ABI: argument validation, workspace layout, launches.  Host code only.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "kvs_internal.cuh"
+
+constexpr int KVS_HOST_CHUNKS = 16;   // the host entry point pipelines copies and kernels over this many chunks
 
 struct kvs_ctx {
   int device = 0;
@@ -18,6 +22,9 @@ struct kvs_ctx {
   bool timing = false;
   bool timed = false;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before the ordering kernel, between, after the builder
+  // host entry point: input copies run on a stream of their own, one event per chunk of instances
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t chunk_ev[KVS_HOST_CHUNKS + 1] = {};
   std::string err;
 };
 
@@ -158,8 +165,12 @@ int check_settings(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* s
   return KVS_OK;
 }
 
+// A call on a sub-range of the instances (host entry point): the `P` settings all name instances in
+// [i0, i1) and are evaluations e0 .. e0 + P - 1 of a batch of P_total; `ev` already points at e0.
+struct FusedRange { int64_t i0, i1, e0, P_total; };
+
 int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P,
-              const kvs_schedule_out* out, const kvs_eval_out* ev, int do_profile) {
+              const kvs_schedule_out* out, const kvs_eval_out* ev, int do_profile, const FusedRange* rg = nullptr) {
   if (!ctx) return KVS_E_STATE;
   int rc = check_instances(ctx, inst);
   if (rc) return rc;
@@ -179,22 +190,25 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   if (P == 0) return KVS_OK;
 
   const int64_t N = inst->n_jobs_total, I = inst->n_instances, max_n = inst->max_jobs_per_instance;
-  const Layout L = make_layout(N, I, max_n, P, false);
+  const Layout L = make_layout(N, I, max_n, rg ? rg->P_total : P, false);
   if (L.total > ctx->workspace_bytes)
     return fail(ctx, KVS_E_CAPACITY, "workspace too small for this call (see kvs_workspace_bytes)");
   cudaError_t ce = cudaSetDevice(ctx->device);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
   unsigned char* ws = ctx->workspace;
-  ce = cudaMemcpyAsync(ws + L.settings, settings, static_cast<size_t>(P) * sizeof(kvs_setting), cudaMemcpyHostToDevice, ctx->stream);
+  const int64_t i0 = rg ? rg->i0 : 0, n_inst = rg ? rg->i1 - rg->i0 : I, e0 = rg ? rg->e0 : 0;
+  unsigned char* const settings_dev = ws + L.settings + static_cast<size_t>(e0) * sizeof(kvs_setting);
+  ce = cudaMemcpyAsync(settings_dev, settings, static_cast<size_t>(P) * sizeof(kvs_setting), cudaMemcpyHostToDevice, ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of settings");
 
   bool need_order = inst->o_est != nullptr;
   for (int64_t e = 0; e < P && !need_order; ++e) need_order = settings[e].family != KVS_GSA;
 
   SortParams sp{};
-  sp.job_off = inst->job_off; sp.s = inst->s; sp.o = inst->o; sp.key = inst->o_est; sp.arrival = inst->arrival;
-  sp.window = inst->window; sp.n_instances = I; sp.max_jobs = max_n; sp.need_order = need_order ? 1 : 0;
-  sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
+  // the ordering kernel numbers its instances from 0: a sub-range shifts the per-instance arrays
+  sp.job_off = inst->job_off + i0; sp.s = inst->s; sp.o = inst->o; sp.key = inst->o_est; sp.arrival = inst->arrival;
+  sp.window = inst->window; sp.n_instances = n_inst; sp.max_jobs = max_n; sp.need_order = need_order ? 1 : 0;
+  sp.stats = reinterpret_cast<InstStats*>(ws + L.stats) + i0;
   sp.perm = reinterpret_cast<int32_t*>(ws + L.perm);
   sp.perm_tmp = reinterpret_cast<int32_t*>(ws + L.perm_tmp);
   sp.iperm = reinterpret_cast<int32_t*>(ws + L.iperm);
@@ -206,23 +220,23 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bool event_form = false;
   if (do_profile && !inst->o_est)
     for (int64_t e = 0; e < P && !event_form; ++e) event_form = settings[e].family >= KVS_SPS;
-  sp.prefix_s = event_form ? reinterpret_cast<i64*>(ws + L.prefix_s) : nullptr;
+  sp.prefix_s = event_form ? reinterpret_cast<i64*>(ws + L.prefix_s) + i0 : nullptr;   // instance j writes at job_off[j] + j
   const int64_t sort_cap = static_cast<int64_t>(ctx->sm_count) * 2;
-  const int sort_grid = static_cast<int>(I < sort_cap ? I : sort_cap);
-  if (ctx->timing) cudaEventRecord(ctx->ev[0], ctx->stream);
+  const int sort_grid = static_cast<int>(n_inst < sort_cap ? n_inst : sort_cap);
+  if (ctx->timing && !rg) cudaEventRecord(ctx->ev[0], ctx->stream);
   ce = kvs_launch_sort(sp, sort_grid, ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "sort launch");
-  if (ctx->timing) cudaEventRecord(ctx->ev[1], ctx->stream);
+  if (ctx->timing && !rg) cudaEventRecord(ctx->ev[1], ctx->stream);
 
   BuildParams bp{};
   bp.job_off = inst->job_off; bp.s = inst->s; bp.o = inst->o; bp.key = inst->o_est; bp.arrival = inst->arrival;
   bp.window = inst->window; bp.n_instances = I; bp.max_jobs = max_n;
   bp.perm = sp.perm; bp.sorted_s = sp.sorted_s; bp.sorted_o = sp.sorted_o; bp.sorted_key = sp.sorted_key;
-  bp.prefix_s = sp.prefix_s;
+  bp.prefix_s = event_form ? reinterpret_cast<i64*>(ws + L.prefix_s) : nullptr;
   bp.iperm = sp.iperm;
   bp.fin_rank = reinterpret_cast<int32_t*>(ws + L.fin_rank);
-  bp.stats = sp.stats;
-  bp.settings = reinterpret_cast<const kvs_setting*>(ws + L.settings);
+  bp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
+  bp.settings = reinterpret_cast<const kvs_setting*>(settings_dev);
   bp.P = P; bp.out = o; bp.ev = v; bp.do_profile = do_profile;
   bp.lists = reinterpret_cast<int32_t*>(ws + L.lists);
   ull* const counters = reinterpret_cast<ull*>(ws + L.counter);
@@ -248,7 +262,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.counter = counters + 2;
   ce = kvs_launch_build(bp, grid_for(ctx->build_ctas_per_sm), ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "build launch");
-  if (ctx->timing) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; }
+  if (ctx->timing && !rg) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; }
   return KVS_OK;
 }
 
@@ -283,8 +297,11 @@ int kvs_init(const kvs_init_params* params, kvs_ctx** out) {
 }
 
 int kvs_destroy(kvs_ctx* ctx) {
-  if (ctx)
+  if (ctx) {
     for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->chunk_ev) if (e) cudaEventDestroy(e);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  }
   delete ctx;
   return KVS_OK;
 }
@@ -347,22 +364,34 @@ int kvs_evaluate_built_host(kvs_ctx* ctx, const kvs_instances* inst, const kvs_s
   if (rc) return rc;
   if (!ev) return fail(ctx, KVS_E_ARG, "eval_out: null");
   if (ev->profile) return fail(ctx, KVS_E_ARG, "host entry point returns scalars only (profile must be NULL)");
-  if (P < 0) return fail(ctx, KVS_E_ARG, "settings: negative count");
+  rc = check_settings(ctx, inst, settings, P);
+  if (rc) return rc;
   const int64_t N = inst->n_jobs_total, I = inst->n_instances;
+  for (int64_t i = 0; i < I; ++i)
+    if (inst->job_off[i] < 0 || inst->job_off[i + 1] < inst->job_off[i] || inst->job_off[i + 1] > N)
+      return fail(ctx, KVS_E_ARG, "instances: job_off is not nondecreasing within [0, n_jobs_total]");
   const Layout L = make_layout(N, I, inst->max_jobs_per_instance, P, true);
   if (L.total > ctx->workspace_bytes) return fail(ctx, KVS_E_CAPACITY, "workspace too small for host staging (see kvs_workspace_bytes)");
   cudaError_t ce = cudaSetDevice(ctx->device);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
+  if (!ctx->copy_stream) {
+    if ((ce = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(ctx, ce, "cudaStreamCreate");
+    for (cudaEvent_t& e : ctx->chunk_ev)
+      if ((ce = cudaEventCreateWithFlags(&e, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(ctx, ce, "cudaEventCreate");
+  }
   unsigned char* ws = ctx->workspace;
-  auto h2d = [&](size_t off, const void* src, size_t bytes) {
-    return (src && bytes) ? cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, ctx->stream) : cudaSuccess;
-  };
-  if ((ce = h2d(L.st_off, inst->job_off, static_cast<size_t>(I + 1) * 8)) != cudaSuccess ||
-      (ce = h2d(L.st_s, inst->s, static_cast<size_t>(N) * 4)) != cudaSuccess ||
-      (ce = h2d(L.st_o, inst->o, static_cast<size_t>(N) * 4)) != cudaSuccess ||
-      (ce = h2d(L.st_key, inst->o_est, static_cast<size_t>(N) * 4)) != cudaSuccess ||
-      (ce = h2d(L.st_arr, inst->arrival, static_cast<size_t>(N) * 8)) != cudaSuccess)
-    return fail_cuda(ctx, ce, "host-to-device copy of the instances");
+
+  // Evaluations are worked off chunk of instances by chunk of instances, so that the copy of the
+  // next chunk's jobs overlaps the kernels of the current one: order them by instance (stable).
+  std::vector<int64_t> order(static_cast<size_t>(P));
+  for (int64_t e = 0; e < P; ++e) order[static_cast<size_t>(e)] = e;
+  bool identity = true;
+  for (int64_t e = 1; e < P && identity; ++e) identity = settings[e - 1].instance <= settings[e].instance;
+  if (!identity)
+    std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return settings[a].instance < settings[b].instance; });
+  std::vector<kvs_setting> sorted(static_cast<size_t>(P));
+  for (int64_t r = 0; r < P; ++r) sorted[static_cast<size_t>(r)] = settings[order[static_cast<size_t>(r)]];
+
   kvs_instances dev = *inst;
   dev.job_off = reinterpret_cast<const int64_t*>(ws + L.st_off);
   dev.s = reinterpret_cast<const int32_t*>(ws + L.st_s);
@@ -377,20 +406,81 @@ int kvs_evaluate_built_host(kvs_ctx* ctx, const kvs_instances* inst, const kvs_s
   d.n_unfinished = reinterpret_cast<int64_t*>(ws + L.sc_unf);
   d.feasible = reinterpret_cast<uint8_t*>(ws + L.sc_feas);
   d.status = reinterpret_cast<int32_t*>(ws + L.sc_stat);
-  rc = run_fused(ctx, &dev, settings, P, nullptr, &d, 1);
-  if (rc) return rc;
-  auto d2h = [&](void* dst, size_t off, size_t bytes) {
-    return (dst && bytes) ? cudaMemcpyAsync(dst, ws + off, bytes, cudaMemcpyDeviceToHost, ctx->stream) : cudaSuccess;
-  };
+
+  // the staging areas may still be read by earlier work on the context's stream
+  if ((ce = cudaEventRecord(ctx->chunk_ev[KVS_HOST_CHUNKS], ctx->stream)) != cudaSuccess ||
+      (ce = cudaStreamWaitEvent(ctx->copy_stream, ctx->chunk_ev[KVS_HOST_CHUNKS], 0)) != cudaSuccess)
+    return fail_cuda(ctx, ce, "stream ordering");
+  ce = cudaMemcpyAsync(ws + L.st_off, inst->job_off, static_cast<size_t>(I + 1) * 8, cudaMemcpyHostToDevice, ctx->copy_stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "host-to-device copy of job_off");
+  const int64_t n_chunks = I < KVS_HOST_CHUNKS ? (I > 0 ? I : 1) : KVS_HOST_CHUNKS;
+  int64_t r0 = 0;
+  for (int64_t c = 0; c < n_chunks; ++c) {
+    const int64_t i0 = c * I / n_chunks, i1 = (c + 1) * I / n_chunks;
+    const int64_t j0 = I ? inst->job_off[i0] : 0, j1 = I ? inst->job_off[i1] : 0;
+    const size_t cnt = static_cast<size_t>(j1 - j0);
+    auto h2d = [&](size_t off, const void* src, size_t elem) {
+      return (src && cnt) ? cudaMemcpyAsync(ws + off + static_cast<size_t>(j0) * elem, static_cast<const unsigned char*>(src) + static_cast<size_t>(j0) * elem,
+                                            cnt * elem, cudaMemcpyHostToDevice, ctx->copy_stream)
+                          : cudaSuccess;
+    };
+    if ((ce = h2d(L.st_s, inst->s, 4)) != cudaSuccess || (ce = h2d(L.st_o, inst->o, 4)) != cudaSuccess ||
+        (ce = h2d(L.st_key, inst->o_est, 4)) != cudaSuccess || (ce = h2d(L.st_arr, inst->arrival, 8)) != cudaSuccess)
+      return fail_cuda(ctx, ce, "host-to-device copy of the instances");
+    if ((ce = cudaEventRecord(ctx->chunk_ev[c], ctx->copy_stream)) != cudaSuccess ||
+        (ce = cudaStreamWaitEvent(ctx->stream, ctx->chunk_ev[c], 0)) != cudaSuccess)
+      return fail_cuda(ctx, ce, "stream ordering");
+    int64_t r1 = r0;
+    while (r1 < P && sorted[static_cast<size_t>(r1)].instance < i1) ++r1;
+    if (r1 > r0) {
+      kvs_eval_out dc = d;
+      dc.peak += r0; dc.flow += r0; dc.job_steps += r0; dc.horizon += r0; dc.n_unfinished += r0; dc.feasible += r0; dc.status += r0;
+      const FusedRange rg{i0, i1, r0, P};
+      rc = run_fused(ctx, &dev, sorted.data() + r0, r1 - r0, nullptr, &dc, 1, &rg);
+      if (rc) return rc;
+    }
+    r0 = r1;
+  }
+
+  // results come back in the order the evaluations were worked off
   const size_t p8 = static_cast<size_t>(P) * 8;
-  if ((ce = d2h(ev->peak, L.sc_peak, p8)) != cudaSuccess || (ce = d2h(ev->flow, L.sc_flow, p8)) != cudaSuccess ||
-      (ce = d2h(ev->job_steps, L.sc_steps, p8)) != cudaSuccess || (ce = d2h(ev->horizon, L.sc_hor, p8)) != cudaSuccess ||
-      (ce = d2h(ev->n_unfinished, L.sc_unf, p8)) != cudaSuccess ||
-      (ce = d2h(ev->feasible, L.sc_feas, static_cast<size_t>(P))) != cudaSuccess ||
-      (ce = d2h(ev->status, L.sc_stat, static_cast<size_t>(P) * 4)) != cudaSuccess)
+  std::vector<int64_t> t64;
+  std::vector<int32_t> t32;
+  std::vector<uint8_t> t8;
+  auto fetch = [&](void* dst, size_t off, size_t elem) -> cudaError_t {
+    if (!dst || P == 0) return cudaSuccess;
+    if (identity) return cudaMemcpyAsync(dst, ws + off, static_cast<size_t>(P) * elem, cudaMemcpyDeviceToHost, ctx->stream);
+    // scattered back through a temporary once the stream has finished
+    return cudaSuccess;
+  };
+  if ((ce = fetch(ev->peak, L.sc_peak, 8)) != cudaSuccess || (ce = fetch(ev->flow, L.sc_flow, 8)) != cudaSuccess ||
+      (ce = fetch(ev->job_steps, L.sc_steps, 8)) != cudaSuccess || (ce = fetch(ev->horizon, L.sc_hor, 8)) != cudaSuccess ||
+      (ce = fetch(ev->n_unfinished, L.sc_unf, 8)) != cudaSuccess || (ce = fetch(ev->feasible, L.sc_feas, 1)) != cudaSuccess ||
+      (ce = fetch(ev->status, L.sc_stat, 4)) != cudaSuccess)
     return fail_cuda(ctx, ce, "device-to-host copy of the results");
   ce = cudaStreamSynchronize(ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "stream synchronize");
+  if (!identity && P > 0) {
+    t64.resize(static_cast<size_t>(P)); t32.resize(static_cast<size_t>(P)); t8.resize(static_cast<size_t>(P));
+    auto back64 = [&](int64_t* dst, size_t off) -> cudaError_t {
+      if (!dst) return cudaSuccess;
+      const cudaError_t e = cudaMemcpy(t64.data(), ws + off, p8, cudaMemcpyDeviceToHost);
+      if (e == cudaSuccess) for (int64_t r = 0; r < P; ++r) dst[order[static_cast<size_t>(r)]] = t64[static_cast<size_t>(r)];
+      return e;
+    };
+    if ((ce = back64(ev->peak, L.sc_peak)) != cudaSuccess || (ce = back64(ev->flow, L.sc_flow)) != cudaSuccess ||
+        (ce = back64(ev->job_steps, L.sc_steps)) != cudaSuccess || (ce = back64(ev->horizon, L.sc_hor)) != cudaSuccess ||
+        (ce = back64(ev->n_unfinished, L.sc_unf)) != cudaSuccess)
+      return fail_cuda(ctx, ce, "device-to-host copy of the results");
+    if (ev->feasible) {
+      if ((ce = cudaMemcpy(t8.data(), ws + L.sc_feas, static_cast<size_t>(P), cudaMemcpyDeviceToHost)) != cudaSuccess) return fail_cuda(ctx, ce, "device-to-host copy of the results");
+      for (int64_t r = 0; r < P; ++r) ev->feasible[order[static_cast<size_t>(r)]] = t8[static_cast<size_t>(r)];
+    }
+    if (ev->status) {
+      if ((ce = cudaMemcpy(t32.data(), ws + L.sc_stat, static_cast<size_t>(P) * 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return fail_cuda(ctx, ce, "device-to-host copy of the results");
+      for (int64_t r = 0; r < P; ++r) ev->status[order[static_cast<size_t>(r)]] = t32[static_cast<size_t>(r)];
+    }
+  }
   return KVS_OK;
 }
 

@@ -167,3 +167,35 @@ def test_int64_times(par):
     assert r64.status.cpu().tolist() == [0] and int(r64.horizon[0]) == S.horizon == 3_000_000_000
     assert np.array_equal(r64.job_completion.cpu().numpy(), S.job_completion) and int(r64.flow[0]) == S.flow
     assert int(r64.peak[0]) == oracle.evaluate_events(S.run_start, S.run_len, S.run_s).peak
+
+
+def test_host_entry_point(par):
+    """kvs_evaluate_built_host (host buffers in, scalars out, copies pipelined with the kernels over chunks of
+    instances) against the oracle, with the evaluations in instance order and in a shuffled order."""
+    import oracle
+    from paper_2601_22996_b200.api import Scheduler
+    cases = [(workloads.config2(n_inst=37, n=1500), 0, ("GBA", "GSA", "SPS", "SIMS")),
+             (workloads.config3(n_inst=5, n=6000), None, ("GBA", "GSA"))]
+    for inst, window, fams in cases:
+        if window is None:
+            window = inst.meta["window"]
+        I = inst.n_instances
+        st = binding.settings_grid(range(I), fams, [inst.meta["M"][len(inst.meta["M"]) // 2]])
+        n = int((inst.job_off[1:] - inst.job_off[:-1]).max())
+        sched = par.scheduler()
+        for order in (np.arange(st.shape[0]), np.random.default_rng(7).permutation(st.shape[0])):
+            s2 = np.ascontiguousarray(st[order])
+            P = s2.shape[0]
+            ctx = sched.context(binding.workspace_bytes(int(inst.s.numel()), I, n, P, host_staging=True))
+            hev = {k: torch.full_like(v, -5, device="cpu").pin_memory() for k, v in Scheduler.scalars(P, "cpu").items()}
+            hin = workloads.Instances(inst.job_off, inst.s.pin_memory(), inst.o.pin_memory(),
+                                      None if inst.o_est is None else inst.o_est.pin_memory(),
+                                      None if inst.arrival is None else inst.arrival.pin_memory())
+            ctx.evaluate_built_host(hin, s2, hev, window=window, max_jobs=n)
+            for e in range(0, P, max(1, P // 40)):
+                S = par.oracle_eval(inst, s2[e], window)
+                assert S.status == 0 and int(hev["status"][e]) == 0
+                assert (int(hev["flow"][e]), int(hev["horizon"][e]), int(hev["job_steps"][e]), int(hev["n_unfinished"][e])) == \
+                       (S.flow, S.horizon, S.job_steps, S.n_unfinished)
+                E = oracle.evaluate_dense(S.run_start, S.run_len, S.run_s, want_profile=False)
+                assert int(hev["peak"][e]) == E.peak and int(hev["feasible"][e]) == int(E.peak <= int(s2[e]["M"]))
