@@ -53,6 +53,7 @@ struct FShared {
   u128 pw_a[MAXP + 1];
   u128 pw_b[MAXP + 1];
   u64 taupre[MAXP + 1];       // sum of tau_q over q < p
+  u64 kinv[MAXP];             // floor(2^64 / k_p) + 1, see slot_mul
   i64 plen[MAXP];
   i64 red64[32];
   i64 next_eval;
@@ -147,6 +148,16 @@ __device__ __forceinline__ int class_pow2(u32 X, u32 v) {
 __device__ __forceinline__ u32 slot32(u32 r, u32 tau, u32 k) {
   const u64 x = static_cast<u64>(r) * tau;
   if ((x >> 32) == 0) return static_cast<u32>(x) / k;
+  return static_cast<u32>(x / k);
+}
+
+// The same with the division replaced by a multiplication: kinv = floor(2^64 / k) + 1 (k >= 2).
+// For x = r * tau below 2^32, x * kinv / 2^64 = x/k + x*e/(k*2^64) with 0 < e <= k; the excess is
+// below 2^-32 while the fractional part of x/k stays at least 1/k > 2^-31 short of the next integer,
+// so the high word of the product is exactly floor(x / k).
+__device__ __forceinline__ u32 slot_mul(u32 r, u32 tau, u32 k, u64 kinv) {
+  const u64 x = static_cast<u64>(r) * tau;
+  if ((x >> 32) == 0) return k == 1 ? static_cast<u32>(x) : static_cast<u32>(__umul64hi(x, kinv));
   return static_cast<u32>(x / k);
 }
 
@@ -888,6 +899,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
         i64 len = 0;
         if (N > 0) len = (sim ? static_cast<i64>(ceil_div_u(N, k) - 1) * tau : static_cast<i64>(static_cast<u64>(N - 1) * tau / k)) + tau;
         sh.plen[tid] = len;
+        sh.kinv[tid] = k >= 2 ? ~0ull / k + 1ull : 0ull;
         // memory is kept modulo 2^32: the general kernel reports evaluations whose bound reaches that
         if ((walk || event_form) && N > 0 && min_i64(N, static_cast<i64>(k) + 1) * (static_cast<i64>(stats.s_max) + tau) >= (static_cast<i64>(1) << 32))
           sh.fallback = 1;
@@ -940,7 +952,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             else fin = oj <= tau0;
             const u32 rank = static_cast<u32>(pos_[u] - seg_lo - sh.ent[ph]);
             const u32 tau = sh.tau[ph], k = sh.k[ph];
-            const u32 stt = sh.pbase[ph] + (sim ? (rank / k) * tau : slot32(rank, tau, k));
+            const u32 stt = sh.pbase[ph] + (sim ? (rank / k) * tau : slot_mul(rank, tau, k, sh.kinv[ph]));
             const u32 d = fin ? oj : tau;
             acc.steps += d;
             acc.hmax = max(acc.hmax, stt + d);
@@ -998,7 +1010,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           if (lane + 64 < pmin) g2 += nvalid;
           if (valid) {
             const u32 tau = sh.tau[l], k = sh.k[l];
-            const u32 stt = sh.pbase[l] + slot32(rank, tau, k);
+            const u32 stt = sh.pbase[l] + slot_mul(rank, tau, k, sh.kinv[l]);
             acc.steps += ov + (sh.taupre[l] - sh.taupre[f]);
             if (keyed) {
               fin_start[seg_lo + x] = stt;
