@@ -53,6 +53,7 @@ def lib():
         L.kvo_phases.argtypes = [p, p, p, p]
         L.kvo_eval_dense.argtypes = [i64, p, p, p, p, i64, p]
         L.kvo_eval_events.argtypes = [i64, p, p, p, p]
+        L.kvo_bounds.argtypes = [i64, p, p, i64, i32, i32, i64, i64, p]
         L.kvo_opt_bruteforce.restype = i64
         L.kvo_opt_bruteforce.argtypes = [i32, i64, p, i64]
         _lib = L
@@ -157,6 +158,23 @@ def evaluate_events(run_start, run_len, run_s) -> Evaluation:
     out = np.zeros(4, dtype=np.int64)
     lib().kvo_eval_events(int(st.shape[0]), _ptr(st), _ptr(ln), _ptr(ss), _ptr(out))
     return Evaluation(int(out[0]), int(out[1]), int(out[2]), -1, None)
+
+
+@dataclass
+class Bounds:
+    status: int
+    upper_gba: int        # GBA flow <= upper_gba
+    upper_gsa: int        # GSA flow <= upper_gsa
+    lower_2m: int         # 2 * M * (lower bound on the optimal flow), see kvo_bounds
+
+
+def bounds(s, o, M, *, alpha=(2, 1), beta0=0, s_bar=-1) -> Bounds:
+    """Bounds computed from the class sizes alone (see ``kvo_bounds``)."""
+    s_, o_ = _arr(s, np.int32), _arr(o, np.int32)
+    out = np.zeros(4, dtype=np.int64)
+    lib().kvo_bounds(int(s_.shape[0]), _ptr(s_), _ptr(o_), int(M), int(alpha[0]), int(alpha[1]), int(beta0),
+                     int(s_bar), _ptr(out))
+    return Bounds(int(out[0]), int(out[1]), int(out[2]), int(out[3]))
 
 
 def opt_bruteforce(s: int, o, M: int) -> int:

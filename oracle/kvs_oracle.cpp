@@ -16,6 +16,10 @@
 //   * Geometric-Batching-Algorithm (GBA)              - Algorithm "Geometric Batching Algorithm"
 //   * Simultaneous-Schedule (SimS)                    - Appendix "Lower Bounds for SimS", batch size B
 //   * optimum without kills or pauses (brute force)   - footnote to the definition of competitive ratio
+//   * bounds from the class sizes                     - Lemma "Area-Based Lower Bound for OPT", Lemma "GBA Upper
+//                                                       Bound via Packing Efficiency" (ladder term, class-prefix
+//                                                       term), Lemma "GSA Upper Bound via Packing Efficiency"
+//                                                       (phase spillover cost, phase-prefix cost)
 //
 // Parity status.  Pinned by the paper: SPS, SimS, Peak, k*, GBA and GSA with
 // exact response lengths, the dense evaluator (Example 1 memory columns, flow
@@ -388,6 +392,70 @@ void kvo_eval_events(int64_t R, const int64_t* start, const int64_t* len, const 
     i = j;
   }
   out[0] = peak; out[1] = T; out[2] = steps; out[3] = -1;
+}
+
+// ---- bounds from the class sizes ---------------------------------------------
+// Class of a job = first p with tau_p >= o (Algorithm GBA); n_p jobs in class p, n_{>p} and n_{>=p}
+// in later / this-or-later classes.  All sums are written out term by term.
+//   ladder term        Q_p = n_p tau_p + sum_{i < n_p} floor(i tau_p / k_p)
+//   class-prefix term  S_p = sum_{q < p} (floor(n_q tau_q / k_q) + tau_q)
+//   UpperGBA           = sum_p (n_p S_p + Q_p)                       (GBA <= UpperGBA)
+//   spillover cost     D_p = ceil(n_{>p} tau_p / k_p)
+//   phase-prefix cost  T_p = sum_{q < p} (floor(n_{>=q} tau_q / k_q) + tau_q)
+//   GSA bound          = sum_p n_p (T_p + D_p) + sum_p Q_p           (GSA <= it)
+//   lower bound        OPT >= sum_p (AreaLB_p / M) (n_p (n_p + 1) / 2 + n_{>p} n_p), AreaLB_p = Area(x_p, s),
+//                      Area(x, s) = s x + x (x + 1) / 2, where every job of class p is longer than x_p.
+// Reading for x_p (the paper takes the real number tau_hat_0 alpha^(p-1)): its integer part, the
+// slice length tau_(p-1) of the ladder, and x_0 = 0; Area is increasing, so the bound stays valid.
+// The lower bound is returned as the integer 2 M (WithinClass + BetweenClasses).
+// out = [status, UpperGBA, GSA bound, 2*M*lower bound]; status 0 ok, 1 infeasible, 2 a value does
+// not fit 63 bits, 3 bad input.
+void kvo_bounds(int64_t n, const int32_t* s, const int32_t* o, int64_t M, int32_t a, int32_t b, int64_t beta0,
+                int64_t s_bar_in, int64_t* out) {
+  out[0] = out[1] = out[2] = out[3] = 0;
+  if (n < 0 || M < 1 || a <= b || b < 1) { out[0] = 3; return; }
+  i64 s_bar = s_bar_in;
+  if (s_bar < 0) { s_bar = 0; for (i64 i = 0; i < n; ++i) s_bar = std::max<i64>(s_bar, s[i]); }
+  const i64 X = M - s_bar;
+  if (X < 1) { out[0] = 1; return; }
+  for (i64 i = 0; i < n; ++i) {
+    if (o[i] < 1 || s[i] < 0) { out[0] = 3; return; }
+    if (o[i] > X) { out[0] = 1; return; }
+  }
+  const std::vector<i64> tau = ladder(X, a, b, beta0);
+  const size_t L = tau.size();
+  if (L == 0) { out[0] = 3; return; }
+  std::vector<i64> k(L), cnt(L, 0);
+  for (size_t p = 0; p < L; ++p) k[p] = kstar(tau[p], s_bar, M);
+  for (i64 i = 0; i < n; ++i) {
+    size_t p = 0;
+    while (tau[p] < o[i]) ++p;            // tau_(L-1) = X >= o_i
+    ++cnt[p];
+  }
+  typedef __int128 big;
+  const big LIMIT = (static_cast<big>(1) << 63) - 1;
+  big upper_gba = 0, gsa = 0, lower = 0;
+  big class_prefix = 0, phase_prefix = 0;   // S_p and T_p, built up phase by phase
+  i64 later = n;                            // n_{>=p}
+  for (size_t p = 0; p < L; ++p) {
+    const big np_ = cnt[p], t = tau[p], kk = k[p];
+    const big n_ge = later, n_gt = later - cnt[p];
+    big Q = np_ * t;
+    for (i64 i = 0; i < cnt[p]; ++i) Q += (static_cast<big>(i) * t) / kk;
+    upper_gba += np_ * class_prefix + Q;
+    const big D = (n_gt * t + kk - 1) / kk;
+    gsa += np_ * (phase_prefix + D) + Q;
+    const big x = p == 0 ? 0 : tau[p - 1];
+    const big area2 = 2 * static_cast<big>(s_bar) * x + x * (x + 1);          // 2 * Area(x, s_bar)
+    lower += area2 * (np_ * (np_ + 1) / 2 + n_gt * np_);
+    class_prefix += (np_ * t) / kk + t;
+    phase_prefix += (n_ge * t) / kk + t;
+    later -= cnt[p];
+    if (upper_gba > LIMIT || gsa > LIMIT || lower > LIMIT) { out[0] = 2; return; }
+  }
+  out[1] = static_cast<i64>(upper_gba);
+  out[2] = static_cast<i64>(gsa);
+  out[3] = static_cast<i64>(lower);
 }
 
 // ---- brute-force optimum (tiny instances, identical prompt length) ----------

@@ -371,3 +371,50 @@ def test_status_codes():
     assert list(S.job_start) == [0, -1, 2] and list(S.job_completion) == [2, -1, 6] and S.flow == 8
     assert list(S.run_len) == [2, 4, 4]                          # order by o: jobs 0, 2, 1
     assert oracle.build_schedule("GBA", [], [], 100).status == 0
+
+
+def test_bounds_worked_example():
+    """Class-size bounds on an instance small enough to work by hand from the lemmas' formulas.
+    M = 10, s = 2 (X = 8), alpha = 2: ladder 1, 2, 4, 8 with k* = 3, 2, 2, 1 (peak-memory lemma);
+    o = 1, 1, 2, 3, 5, 8 gives class sizes 2, 1, 1, 2.
+      ladder terms Q = 2, 2, 4, 24; class-prefix terms S = 0, 1, 4, 10; UpperGBA = 2 + 3 + 8 + 44 = 57
+      spillover D = 2, 3, 4, 0; phase-prefix T = 0, 3, 9, 19; GSA bound = 4 + 6 + 13 + 38 + 32 = 93
+      2*Area(x, 2) for x = 0, 1, 2, 4 is 0, 6, 14, 36 with weights 11, 4, 3, 3: 2*M*lower = 174."""
+    B = oracle.bounds([2] * 6, [1, 1, 2, 3, 5, 8], 10)
+    assert (B.status, B.upper_gba, B.upper_gsa, B.lower_2m) == (0, 57, 93, 174)
+    assert [int(x) for x in oracle.build_schedule("GBA", [2] * 6, [1, 1, 2, 3, 5, 8], 10).k] == [3, 2, 2, 1]
+    # the order of the jobs does not matter, only the class sizes do
+    assert oracle.bounds([2] * 6, [8, 1, 5, 2, 1, 3], 10) == B
+    assert oracle.bounds([2], [9], 10).status == 1 and oracle.bounds([2], [0], 10).status == 3
+
+
+def test_bounds_hold_for_schedules_and_optimum():
+    """GBA <= UpperGBA and GSA <= its bound (the two packing-efficiency lemmas), the aggregate
+    inequality between the two bounds, and lower bound <= optimum <= every schedule."""
+    rng = np.random.default_rng(55)
+    for alpha in [(2, 1), (3, 2), (4, 3), (7, 4)]:
+        al = Fraction(*alpha)
+        for _ in range(60):
+            s, o, M = _random_instance(rng, hetero=False)
+            B = oracle.bounds(s, o, M, alpha=alpha)
+            gba = oracle.build_schedule("GBA", s, o, M, alpha=alpha)
+            gsa = oracle.build_schedule("GSA", s, o, M, alpha=alpha)
+            assert B.status == 0 and gba.flow <= B.upper_gba and gsa.flow <= B.upper_gsa
+            assert B.upper_gba <= B.upper_gsa <= (2 + 2 / (al - 1)) * B.upper_gba
+            for S in (gba, gsa, oracle.build_schedule("SPS", s, o, M), oracle.build_schedule("SIMS", s, o, M)):
+                assert B.lower_2m <= 2 * M * S.flow
+    for _ in range(60):
+        n, s = int(rng.integers(1, 8)), int(rng.integers(0, 6))
+        o = rng.integers(1, 7, n)
+        M = int(s + o.max() + rng.integers(0, 14))
+        opt = oracle.opt_bruteforce(s, o, M)
+        for alpha in [(2, 1), (3, 2)]:
+            B = oracle.bounds([s] * n, o, M, alpha=alpha)
+            assert B.lower_2m <= 2 * M * opt <= 2 * M * B.upper_gba
+    # a tunable initial slice changes the ladder, not the validity of the upper bounds
+    for _ in range(30):
+        s, o, M = _random_instance(rng, hetero=False)
+        b0 = int(rng.integers(1, 6))
+        B = oracle.bounds(s, o, M, beta0=b0)
+        assert oracle.build_schedule("GBA", s, o, M, beta0=b0).flow <= B.upper_gba
+        assert oracle.build_schedule("GSA", s, o, M, beta0=b0).flow <= B.upper_gsa
