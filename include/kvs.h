@@ -214,6 +214,34 @@ int kvs_evaluate_schedule_noalloc(int32_t device, void* stream, const kvs_runs* 
                                   const kvs_eval_out* ev, int64_t capacity_total,
                                   char* err, uint64_t err_len);
 
+/* Bounds that depend on an instance only through the sizes of its classes (class of a job = first
+ * slice of the ladder that is at least its response length), per (instance, setting):
+ *   upper_gba  UpperGBA, the sum of class-prefix and ladder terms (Lemma "GBA Upper Bound via Packing
+ *              Efficiency"): the GBA schedule's total flow time is at most this;
+ *   upper_gsa  the bound of Lemma "GSA Upper Bound via Packing Efficiency" (phase-prefix cost,
+ *              phase spillover cost, ladder terms);
+ *   lower_2m   2 * M * (WithinClass + BetweenClasses) of Lemma "Area-Based Lower Bound for OPT", an
+ *              integer: the optimal total flow time is at least lower_2m / (2 M).  The memory-time
+ *              area of class p is taken at the integer threshold x_p = tau_(p-1) (x_0 = 0) and at
+ *              the prompt length s_bar of the setting, so the bound is the lemma's for instances
+ *              with one prompt length and a valid, slightly weaker one otherwise when s_bar does
+ *              not exceed any prompt length.
+ * Each DEVICE array has P entries; any may be NULL.  status[] holds kvs_eval_status bits
+ * (KVS_EVAL_RANGE: a value does not fit 63 bits); the three values are -1 unless status is 0. */
+typedef struct {
+  int64_t* upper_gba;
+  int64_t* upper_gsa;
+  int64_t* lower_2m;
+  int32_t* status;
+} kvs_bounds_out;
+
+/* Uses instance, M, alpha_num/alpha_den, beta0 and s_bar of each setting (HOST array of P entries,
+ * copied to the workspace asynchronously); the family, tau and k are ignored.  The instances must
+ * be offline (window = 0); estimates, if present, are ignored: the bounds are statements about the
+ * exact response lengths.  Asynchronous on the context's stream. */
+int kvs_bounds(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P,
+               const kvs_bounds_out* out);
+
 /* Parameter sweep on one instance: SPS or SIMS for every (tau, k) of a grid, scalars only. */
 typedef struct {
   int64_t instance;

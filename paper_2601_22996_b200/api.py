@@ -130,6 +130,19 @@ class Scheduler:
         return Result(ev["status"], ev["flow"], ev["peak"], ev["horizon"], ev["job_steps"], ev["n_unfinished"],
                       ev["feasible"], profile_off=poff, profile=ev.get("profile"))
 
+    def bounds(self, inst: Instances, settings: np.ndarray) -> dict:
+        """Class-size bounds (kvs_bounds) of P (instance, setting) pairs; returns device tensors [P]."""
+        dev = inst.s.device
+        N, I, max_n, _ = self._sizes(inst)
+        P = int(settings.shape[0])
+        if P and (settings["instance"].min() < 0 or settings["instance"].max() >= I):
+            raise binding.KvsError(-1, "settings: instance out of range")
+        ctx = self.context(binding.workspace_bytes(N, I, max_n, P))
+        out = {f: torch.zeros(P, dtype=torch.int64, device=dev) for f in ("upper_gba", "upper_gsa", "lower_2m")}
+        out["status"] = torch.zeros(P, dtype=torch.int32, device=dev)
+        ctx.bounds(inst, settings, out, max_jobs=max_n)
+        return out
+
     def sweep(self, inst: Instances, instance: int, family, M: int, tau, k) -> dict:
         """SPS / SimS over a (tau, k) grid on one instance; returns device tensors [n_tau, n_k]."""
         dev = inst.s.device

@@ -70,9 +70,13 @@ class _SweepOut(Structure):
                 ("job_steps", c_void_p), ("feasible", c_void_p)]
 
 
+class _BoundsOut(Structure):
+    _fields_ = [("upper_gba", c_void_p), ("upper_gsa", c_void_p), ("lower_2m", c_void_p), ("status", c_void_p)]
+
+
 EXPORTS = ["kvs_init", "kvs_destroy", "kvs_last_error", "kvs_set_timing", "kvs_last_timing", "kvs_workspace_bytes",
            "kvs_build_schedule", "kvs_evaluate_built", "kvs_evaluate_built_host", "kvs_evaluate_schedule", "kvs_sweep",
-           "kvs_evaluate_schedule_noalloc"]
+           "kvs_evaluate_schedule_noalloc", "kvs_bounds"]
 
 _lib = None
 
@@ -98,6 +102,7 @@ def load(path: str | None = None):
         L.kvs_evaluate_built_host.argtypes = [c_void_p, POINTER(_Instances), c_void_p, c_int64, POINTER(_EvalOut)]
         L.kvs_evaluate_schedule.argtypes = [c_void_p, POINTER(_Runs), POINTER(_EvalOut)]
         L.kvs_sweep.argtypes = [c_void_p, POINTER(_Instances), POINTER(_SweepParams), POINTER(_SweepOut)]
+        L.kvs_bounds.argtypes = [c_void_p, POINTER(_Instances), c_void_p, c_int64, POINTER(_BoundsOut)]
         L.kvs_evaluate_schedule_noalloc.argtypes = [c_int32, c_void_p, POINTER(_Runs), POINTER(_EvalOut), c_int64,
                                                     ctypes.c_char_p, c_uint64]
         _lib = L
@@ -242,6 +247,15 @@ class Context:
         settings = np.ascontiguousarray(settings, dtype=SETTING_DTYPE)
         self._check(self._lib.kvs_evaluate_built_host(self._ctx, ctypes.byref(ci), settings.ctypes.data_as(c_void_p),
                                                       settings.shape[0], ctypes.byref(eo)))
+
+    def bounds(self, inst: Instances, settings: np.ndarray, out: dict, max_jobs: int | None = None):
+        """kvs_bounds: ``out`` maps upper_gba, upper_gsa, lower_2m (int64 [P]) and status (int32 [P]) to CUDA tensors."""
+        ci = self._instances(inst, 0, max_jobs)
+        bo = _BoundsOut(*[_p(out.get(f[0])) for f in _BoundsOut._fields_])
+        settings = np.ascontiguousarray(settings, dtype=SETTING_DTYPE)
+        self._keep = (settings, inst, out)
+        self._check(self._lib.kvs_bounds(self._ctx, ctypes.byref(ci), settings.ctypes.data_as(c_void_p), settings.shape[0],
+                                         ctypes.byref(bo)))
 
     def evaluate_schedule(self, runs: dict, ev: dict):
         """kvs_evaluate_schedule: ``runs`` maps run_off, run_start, run_len, run_s [, run_flow, M]."""

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libkvs.so")
-SOURCES = ["kvs_api.cu", "kvs_sort.cu", "kvs_build.cu", "kvs_fused.cu", "kvs_generic.cu", "kvs_sweep.cu"]
+SOURCES = ["kvs_api.cu", "kvs_sort.cu", "kvs_build.cu", "kvs_fused.cu", "kvs_bounds.cu", "kvs_generic.cu", "kvs_sweep.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", _INCLUDE, "-I", _CSRC]
 

@@ -514,6 +514,42 @@ int kvs_evaluate_schedule(kvs_ctx* ctx, const kvs_runs* runs, const kvs_eval_out
   return KVS_OK;
 }
 
+int kvs_bounds(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settings, int64_t P, const kvs_bounds_out* out) {
+  if (!ctx) return KVS_E_STATE;
+  int rc = check_instances(ctx, inst);
+  if (rc) return rc;
+  if (!out) return fail(ctx, KVS_E_ARG, "bounds: out is null");
+  if (inst->window != 0) return fail(ctx, KVS_E_ARG, "bounds: needs offline instances (window = 0)");
+  // the family is not used: check the settings as geometric ones
+  std::vector<kvs_setting> geo(settings, settings + (settings && P > 0 ? P : 0));
+  for (kvs_setting& s : geo) { s.family = KVS_GBA; s.tau = 0; s.k = 0; }
+  rc = check_settings(ctx, inst, P > 0 ? geo.data() : settings, P);
+  if (rc) return rc;
+  if (P == 0) return KVS_OK;
+  const int64_t N = inst->n_jobs_total, I = inst->n_instances, max_n = inst->max_jobs_per_instance;
+  const Layout L = make_layout(N, I, max_n, P, false);
+  if (L.total > ctx->workspace_bytes) return fail(ctx, KVS_E_CAPACITY, "workspace too small for this call (see kvs_workspace_bytes)");
+  cudaError_t ce = cudaSetDevice(ctx->device);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaSetDevice");
+  unsigned char* ws = ctx->workspace;
+  ce = cudaMemcpyAsync(ws + L.settings, geo.data(), static_cast<size_t>(P) * sizeof(kvs_setting), cudaMemcpyHostToDevice, ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of settings");
+  // statistics and validation of the instances (largest prompt and response, input checks): the
+  // ordering kernel without the ordering
+  SortParams sp{};
+  sp.job_off = inst->job_off; sp.s = inst->s; sp.o = inst->o; sp.key = nullptr; sp.arrival = nullptr;
+  sp.window = 0; sp.n_instances = I; sp.max_jobs = max_n; sp.need_order = 0;
+  sp.stats = reinterpret_cast<InstStats*>(ws + L.stats);
+  const int64_t sort_cap = static_cast<int64_t>(ctx->sm_count) * 2;
+  ce = kvs_launch_sort(sp, static_cast<int>(I < sort_cap ? I : sort_cap), ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "statistics launch");
+  const int64_t cap = static_cast<int64_t>(ctx->sm_count) * 8;
+  ce = kvs_launch_bounds(inst->job_off, inst->o, sp.stats, reinterpret_cast<const kvs_setting*>(ws + L.settings), P, *out,
+                         static_cast<int>(P < cap ? P : cap), ctx->stream);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "bounds launch");
+  return KVS_OK;
+}
+
 int kvs_sweep(kvs_ctx* ctx, const kvs_instances* inst, const kvs_sweep_params* params, const kvs_sweep_out* out) {
   if (!ctx) return KVS_E_STATE;
   int rc = check_instances(ctx, inst);

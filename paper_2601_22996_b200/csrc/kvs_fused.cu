@@ -26,6 +26,7 @@
 // An evaluation whose times reach 2^31 or whose memory bound reaches 2^32 is not finished here: its
 // index is appended to a list that the general kernel works off afterwards.
 #include "kvs_events.cuh"
+#include "kvs_ladder.cuh"
 
 namespace {
 
@@ -40,8 +41,6 @@ constexpr int RINGW = 2 * TILE + (2 * TILE) / 8;
 constexpr int GCOL = 2049;
 static_assert((TILE & (TILE - 1)) == 0 && ITEMS % 4 == 0 && ITEMS <= 32 && 32 % ITEMS == 0, "tile layout");
 constexpr u32 TIME_LIMIT = 0x7fffffffu - 4u * TILE;   // phase ends stay below this
-
-typedef unsigned __int128 u128;
 
 struct FShared {
   // two-tile ring of difference arrays: constant terms and slopes.  Round e of the ring (0 <= e <
@@ -67,82 +66,6 @@ struct FShared {
   int ent[MAXP + 1];          // class boundaries in key order
   int n_phases, seg_end, fallback;
 };
-
-__device__ __forceinline__ u32 gcd_u32(u32 x, u32 y) {
-  while (y) { const u32 t = x % y; x = y; y = t; }
-  return x;
-}
-
-// Largest k >= 1 with s*k + (tau*k + tau + k - gcd(tau, k))/2 <= M, given s + tau <= M: the
-// condition reads k*(2s+tau+1) <= 2M - tau + gcd(tau,k), and 1 <= gcd <= tau leaves k0 or k0 + 1
-// with k0 = floor((2M - tau + 1) / (2s + tau + 1)).
-__device__ u32 max_parallelism32(u32 tau, u32 s, u32 M) {
-  const u64 D = 2ull * s + tau + 1ull;
-  const u64 num = 2ull * M - tau + 1ull;
-  u64 k0, r;
-  divmod_u(num, D, &k0, &r);
-  const u64 k1 = k0 + 1;
-  if (k1 >> 31) return static_cast<u32>(k0);
-  return (k1 * D <= 2ull * M - tau + gcd_u32(tau, static_cast<u32>(k1))) ? static_cast<u32>(k1) : static_cast<u32>(k0);
-}
-
-__device__ void ladder32(FShared& sh, i64 X, int a, int b, i64 beta0, u32 s_bar, u32 M) {
-  const int lane = lane_id();
-  if (beta0 <= 0) {
-    if (lane == 0) {
-      u128 pa = 1, pb = 1;
-      int ell = 0;
-      sh.pw_a[0] = 1; sh.pw_b[0] = 1;
-      while (ell + 1 < MAXP + 1) {
-        const u128 na = pa * static_cast<u128>(a), nb = pb * static_cast<u128>(b);
-        if (na > static_cast<u128>(X) * nb) break;
-        pa = na; pb = nb; ++ell;
-        sh.pw_a[ell] = pa; sh.pw_b[ell] = pb;
-      }
-      sh.n_phases = (ell + 1 <= MAXP) ? ell + 1 : 0;
-    }
-    __syncwarp();
-    const int L = sh.n_phases;
-    for (int p = lane; p < L; p += 32) {
-      const int j = L - 1 - p;  // tau_p = floor(X * b^j / a^j)
-      const u32 t = (a == 2 && b == 1) ? static_cast<u32>(X >> j)
-                                       : static_cast<u32>(static_cast<u128>(X) * sh.pw_b[j] / sh.pw_a[j]);
-      sh.tau[p] = t;
-      sh.k[p] = max_parallelism32(t, s_bar, M);
-    }
-  } else {
-    if (lane == 0) {
-      u128 pa = 1, pb = 1;
-      int p = 0;
-      for (;; ++p) {
-        if (p >= MAXP) { p = -1; break; }
-        const u128 num = static_cast<u128>(beta0) * pa;   // tau_p = min(floor(beta0 * a^p / b^p), X)
-        const u32 t = (num >= static_cast<u128>(X) * pb) ? static_cast<u32>(X) : static_cast<u32>(num / pb);
-        sh.tau[p] = t;
-        sh.k[p] = max_parallelism32(t, s_bar, M);
-        if (t >= X) break;
-        pa *= static_cast<u128>(a); pb *= static_cast<u128>(b);
-      }
-      sh.n_phases = p + 1;
-    }
-  }
-  __syncwarp();
-}
-
-// class(v) = first p with tau_p >= v (tau is nondecreasing and tau_(L-1) >= v)
-__device__ __forceinline__ int class_of(const u32* tau, int L, u32 v) {
-  int a = 0, b = L - 1;
-  while (a < b) { const int m = (a + b) >> 1; if (tau[m] >= v) b = m; else a = m + 1; }
-  return a;
-}
-
-// The same for the ladder of alpha = 2, tau_p = X >> (ell - p) with ell = floor(log2 X): the largest
-// shift j with (X >> j) >= v is the difference of the bit lengths, or one less.  1 <= v <= X.
-__device__ __forceinline__ int class_pow2(u32 X, u32 v) {
-  const int j0 = __clz(v) - __clz(X);
-  const int j = (X >> j0) >= v ? j0 : j0 - 1;
-  return (31 - __clz(X)) - j;
-}
 
 // floor(r * tau / k) for r, tau, k below 2^31 with a result below 2^31
 __device__ __forceinline__ u32 slot32(u32 r, u32 tau, u32 k) {

@@ -122,6 +122,8 @@ int kvs_build_ctas_per_sm();
 cudaError_t kvs_launch_fused(const BuildParams& p, int grid, cudaStream_t stream);
 int kvs_fused_ctas_per_sm();
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
+cudaError_t kvs_launch_bounds(const i64* job_off, const int32_t* o, const InstStats* stats, const kvs_setting* settings,
+                              i64 P, const kvs_bounds_out& out, int grid, cudaStream_t stream);
 cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,
                               i64* prefix_o, cudaStream_t stream);
 cudaError_t kvs_launch_sweep(const SweepParams& p, i64* acc_peak, u64* acc_flow, cudaStream_t stream);
