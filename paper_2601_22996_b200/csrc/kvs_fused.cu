@@ -491,6 +491,51 @@ __device__ __forceinline__ void insert_far_ends_list(FShared& sh, const PhaseVie
   }
 }
 
+// A phase in which every position of the window takes part and none completes (index order, all
+// response lengths beyond the slice: the early phases of the slicing algorithm) needs no visit of
+// its runs.  Rank = position, every run lasts tau rounds, so the events of a round are sums over
+// position ranges: with PS[x] = sum of (s + 1) over positions below x and B(u) = number of ranks that
+// start in round u or earlier = min(N, ceil((u + 1) k / tau)), the runs that start in round u add
+// (PS[B(u)] - PS[B(u-1)] - cnt (base + u), cnt) there and the opposite tau rounds later.  Each thread
+// forms the events of its own ITEMS rounds of the tile - starts at u and ends of the runs started
+// at u - tau - and adds them to its own words of the ring: no atomics, no dependence on the number
+// of runs.  u0 = offset of the tile's origin inside the phase.
+__device__ __forceinline__ void pure_phase_events(FShared& sh, const PhaseView& P, const u32* __restrict__ PS, int N, int u0, int buf) {
+  const int e0 = ITEMS * static_cast<int>(threadIdx.x);
+  const int w0 = ring(buf, e0);
+  const u32 tau = P.tau, k = P.k;
+  const u32 kq = k / tau, kr = k - kq * tau;          // k = kq * tau + kr
+#pragma unroll
+  for (int stream = 0; stream < 2; ++stream) {
+    // stream 0: runs that start in the thread's rounds; stream 1: runs that end there (started tau earlier)
+    const i64 ufirst = static_cast<i64>(u0) + e0 - (stream ? static_cast<i64>(tau) : 0);   // start round of the first event
+    // B(ufirst - 1) by one division, then stepped: (u + 1) k = Q tau + R
+    u64 Q = 0, R = 0;
+    i64 u = ufirst - 1;
+    if (u >= 0) divmod_u(static_cast<u64>(u + 1) * k, tau, &Q, &R);
+    u32 b_prev = u >= 0 ? static_cast<u32>(min(static_cast<u64>(N), Q + (R > 0))) : 0u;
+    u32 ps_prev = PS[b_prev];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+      ++u;
+      if (u == 0) { Q = kq; R = kr; }                  // (0 + 1) k
+      else if (u > 0) { Q += kq; R += kr; if (R >= tau) { R -= tau; ++Q; } }
+      const i64 land = u + (stream ? static_cast<i64>(tau) : 0);          // round the event lands in
+      if (u >= 0 && land < static_cast<i64>(P.len)) {
+        const u32 b = static_cast<u32>(min(static_cast<u64>(N), Q + (R > 0)));
+        if (b != b_prev) {
+          const u32 ps = PS[b];
+          const u32 cnt = b - b_prev;
+          const u32 c = (ps - ps_prev) - cnt * (P.base + static_cast<u32>(u));
+          if (stream == 0) { sh.dA[w0 + i] += c; sh.dB[w0 + i] += cnt; }
+          else { sh.dA[w0 + i] -= c; sh.dB[w0 + i] -= cnt; }
+          b_prev = b; ps_prev = ps;
+        }
+      }
+    }
+  }
+}
+
 // Slices longer than a tile: ends that land two or more tiles after the run's start were not
 // inserted when the run was visited; pick them up when their tile comes.  u0 = offset of this
 // tile's origin inside the phase, a0 = the same for the phase's first tile (0 or slightly negative).
@@ -1064,6 +1109,43 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
         uint2* cur = list0;
         uint2* nxt = list1;
         int C = 0;
+        // index order without estimates: the phases before the first class that holds a job are
+        // walked from prefix sums of s + 1 over the positions (see pure_phase_events)
+        int n_pure = 0;
+        u32* const PS = reinterpret_cast<u32*>(list1);
+        if (carry && !est) {
+          while (n_pure + 1 < L && static_cast<int>(G[nsegs * L + n_pure + 1]) == nseg) ++n_pure;
+          if (n_pure > 0) {
+            u32 run = 0;
+            for (int x0 = 0; x0 <= nseg; x0 += T * 4) {
+              const int x = x0 + 4 * tid;
+              u32 v[4], tot = 0;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) { v[j] = tot; if (x + j < nseg) tot += static_cast<u32>(__ldg(S_ord + seg_lo + x + j)) + 1u; }
+              u32 incl = tot;
+#pragma unroll
+              for (int d = 1; d < 32; d <<= 1) {
+                const u32 y = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += y;
+              }
+              __syncthreads();
+              if (lane == 31) sh.redA[warp] = incl;
+              __syncthreads();
+              const u32 w = lane < WARPS ? sh.redA[lane] : 0u;
+              u32 wi = w;
+#pragma unroll
+              for (int d = 1; d < 32; d <<= 1) {
+                const u32 y = __shfl_up_sync(0xffffffffu, wi, d);
+                if (lane >= d) wi += y;
+              }
+              const u32 off = run + __shfl_sync(0xffffffffu, wi - w, warp) + (incl - tot);
+              run += __shfl_sync(0xffffffffu, wi, 31);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) if (x + j <= nseg) PS[x + j] = off + v[j];
+            }
+            __syncthreads();
+          }
+        }
         for (int ph = 0; ph < L; ++ph) {
           const int N = static_cast<int>(sh.np[ph]);
           if (N == 0) continue;
@@ -1124,12 +1206,13 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
             }
             cq += dq; cr += dr;
             if (cr >= utau) { cr -= utau; ++cq; }
-            if (sim) visit_runs<true, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
+            if (ph < n_pure) pure_phase_events(sh, P, PS, N, u0, buf);
+            else if (sim) visit_runs<true, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             else if (list_mode) C_next = visit_list(sh, P, V, nxt, C_next, r_next, r_b, u0, buf, dense);
             else if (carry) visit_runs<false, true>(sh, P, r_next, r_b, u0, buf, dense, combine);
             else visit_runs<false, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             r_next = r_b;
-            if (P.tau > TILE) {
+            if (P.tau > TILE && ph >= n_pure) {
               if (list_mode) insert_far_ends_list(sh, P, V, N, a0, u0, wlen, buf);
               else if (carry) insert_far_ends<true>(sh, P, sim, N, a0, u0, wlen, buf);
               else insert_far_ends<false>(sh, P, sim, N, a0, u0, wlen, buf);
