@@ -26,10 +26,10 @@ from paper_2601_22996_b200 import workloads  # noqa: E402
 
 METRIC, UNIT = "schedule_evaluation_job_steps_per_sec", "job-steps/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_fused_eval launch, from the ncu capture summarised in
-# profiles/k_fused_eval_c5.md (592 instances of config 5, all four families: 2,368 evaluations, 4.728 GB).
+# profiles/k_fused_eval_c5.md (592 instances of config 5, all four families: 2,368 evaluations, 4.685 GB).
 # Traffic grows with the number of evaluations (each CTA works on one at a time), so a launch is scaled
 # by its evaluation count.  Valid for the kernel state named in that file; set to None when the kernel changes.
-C5_TRAFFIC_BYTES_PER_EVALUATION = 4.727948e9 / 2368
+C5_TRAFFIC_BYTES_PER_EVALUATION = 4.684714e9 / 2368
 WORKLOADS = {
     # name: (generator, instances, jobs per instance, families, description)
     "c2": ("config2", 1024, 10_000, ["GBA", "GSA"], "config 2: 1,024 instances x 10,000 jobs, M in {2^17..2^24}, GBA+GSA"),
