@@ -171,7 +171,7 @@ int kvs_evaluate_built(kvs_ctx* ctx, const kvs_instances* inst, const kvs_settin
  * (and o_est, arrival) to the workspace, runs the fused path, and copies the per-evaluation
  * scalars back.  Every pointer of `inst` and of `ev` is a HOST pointer here (pinned memory
  * makes the copies asynchronous); `ev->profile` must be NULL.  The instances are worked off in up
- * to 16 chunks: the jobs of the next chunk are copied on a second stream while the kernels of the
+ * to 16 chunks (of about a thousand evaluations or more, so small batches stay in one piece): the jobs of the next chunk are copied on a second stream while the kernels of the
  * current one run, so the settings may come in any order but are evaluated grouped by instance
  * (results are returned in the caller's order).  job_off is read on the host and must be
  * nondecreasing.  The call returns after the stream has been synchronised. */

@@ -413,7 +413,11 @@ int kvs_evaluate_built_host(kvs_ctx* ctx, const kvs_instances* inst, const kvs_s
     return fail_cuda(ctx, ce, "stream ordering");
   ce = cudaMemcpyAsync(ws + L.st_off, inst->job_off, static_cast<size_t>(I + 1) * 8, cudaMemcpyHostToDevice, ctx->copy_stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "host-to-device copy of job_off");
-  const int64_t n_chunks = I < KVS_HOST_CHUNKS ? (I > 0 ? I : 1) : KVS_HOST_CHUNKS;
+  // a chunk should still fill the GPU: about a thousand evaluations each, at most KVS_HOST_CHUNKS chunks
+  int64_t n_chunks = P / 1024;
+  if (n_chunks > KVS_HOST_CHUNKS) n_chunks = KVS_HOST_CHUNKS;
+  if (n_chunks > I) n_chunks = I;
+  if (n_chunks < 1) n_chunks = 1;
   int64_t r0 = 0;
   for (int64_t c = 0; c < n_chunks; ++c) {
     const int64_t i0 = c * I / n_chunks, i1 = (c + 1) * I / n_chunks;
