@@ -19,6 +19,7 @@ struct kvs_ctx {
   int sm_count = 0;
   int build_ctas_per_sm = 1;
   int fused_ctas_per_sm = 1;
+  int light_ctas_per_sm = 1;
   bool timing = false;
   bool timed = false;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before the ordering kernel, between, after the builder
@@ -48,7 +49,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // one stream, so the entry points reuse the workspace from offset 0; the layout without staging
 // is a prefix of the layout with staging.
 struct Layout {
-  size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter, slow_list;
+  size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter, slow_list, walk_list, light_list;
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -70,8 +71,10 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
   L.lists = take(static_cast<size_t>(grid) * static_cast<size_t>(KVS_CTA_SCRATCH(max_n)));
   L.fin_rank = take(static_cast<size_t>(grid) * static_cast<size_t>(max_n) * 4);
-  L.counter = take(32);   // work counter of the fast kernel, length of its left-over list, work counter of the general kernel
+  L.counter = take(64);   // work counters of the three kernels, lengths of the two hand-over lists
   L.slow_list = take(static_cast<size_t>(P) * 8);
+  L.walk_list = take(static_cast<size_t>(P) * 8);
+  L.light_list = take(static_cast<size_t>(P) * 8);
   if (staging) {
     L.st_off = take(static_cast<size_t>(I + 1) * 8);
     L.st_s = take(static_cast<size_t>(N) * 4);
@@ -251,10 +254,36 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   // come back in a list that the general kernel works off.  Other calls go to the general kernel.
   const bool fast = !run_out && !o.job_start64 && !o.job_completion64;
   if (fast) {
-    bp.counter = counters;
+    // Two variants of the fast kernel.  The light one (no ring, three CTAs per SM) takes the
+    // evaluations that walk no rounds: all of them when no profile is formed, else the SPS / SimS
+    // ones, of which it passes on those that turn out to want their profile.  The full one takes
+    // the geometric evaluations, listed here on the host, and what the light one passed on.
+    std::vector<int64_t> ids(static_cast<size_t>(P));
+    int64_t n_full = 0, n_light = 0;
+    for (int64_t e = 0; e < P; ++e)
+      if (do_profile && settings[e].family <= KVS_GSA) ids[static_cast<size_t>(n_full++)] = e;
+    for (int64_t e = 0; e < P; ++e)
+      if (!(do_profile && settings[e].family <= KVS_GSA)) ids[static_cast<size_t>(n_full + n_light++)] = e;
+    const unsigned long long init[8] = {0, 0, 0, static_cast<unsigned long long>(n_full), 0, static_cast<unsigned long long>(n_light), 0, 0};
+    if ((ce = cudaMemcpyAsync(counters, init, sizeof(init), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+        (n_full && (ce = cudaMemcpyAsync(ws + L.walk_list, ids.data(), static_cast<size_t>(n_full) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) ||
+        (n_light && (ce = cudaMemcpyAsync(ws + L.light_list, ids.data() + n_full, static_cast<size_t>(n_light) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess))
+      return fail_cuda(ctx, ce, "copy of the evaluation lists");
     bp.slow_count = counters + 1;
     bp.slow_list = reinterpret_cast<i64*>(ws + L.slow_list);
-    ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), ctx->stream);
+    bp.walk_count = counters + 3;
+    bp.walk_list = reinterpret_cast<i64*>(ws + L.walk_list);
+    if (n_light) {
+      bp.counter = counters;
+      bp.eval_list = reinterpret_cast<const i64*>(ws + L.light_list);
+      bp.eval_count = counters + 5;
+      ce = kvs_launch_fused(bp, grid_for(ctx->light_ctas_per_sm), 1, ctx->stream);
+      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    }
+    bp.counter = counters + 4;
+    bp.eval_list = bp.walk_list;
+    bp.eval_count = bp.walk_count;
+    ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, ctx->stream);
     if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
     bp.eval_list = bp.slow_list;
     bp.eval_count = bp.slow_count;
@@ -291,7 +320,8 @@ int kvs_init(const kvs_init_params* params, kvs_ctx** out) {
   }
   ctx->sm_count = prop.multiProcessorCount;
   ctx->build_ctas_per_sm = kvs_build_ctas_per_sm();
-  ctx->fused_ctas_per_sm = kvs_fused_ctas_per_sm();
+  ctx->fused_ctas_per_sm = kvs_fused_ctas_per_sm(0);
+  ctx->light_ctas_per_sm = kvs_fused_ctas_per_sm(1);
   *out = ctx;
   return KVS_OK;
 }

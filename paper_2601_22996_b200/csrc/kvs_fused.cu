@@ -25,6 +25,8 @@
 //
 // An evaluation whose times reach 2^31 or whose memory bound reaches 2^32 is not finished here: its
 // index is appended to a list that the general kernel works off afterwards.
+#include <cstddef>
+
 #include "kvs_events.cuh"
 #include "kvs_ladder.cuh"
 
@@ -43,12 +45,6 @@ static_assert((TILE & (TILE - 1)) == 0 && ITEMS % 4 == 0 && ITEMS <= 32 && 32 % 
 constexpr u32 TIME_LIMIT = 0x7fffffffu - 4u * TILE;   // phase ends stay below this
 
 struct FShared {
-  // two-tile ring of difference arrays: constant terms and slopes.  Round e of the ring (0 <= e <
-  // 2*TILE) lives at word e + 4*(e/32): four spare words after every 32 keep the 16-byte loads of
-  // the scan (a thread owns ITEMS consecutive rounds) free of bank conflicts while the index of an
-  // event stays a shift and an add.
-  u32 dA[RINGW];
-  u32 dB[RINGW];
   u128 pw_a[MAXP + 1];
   u128 pw_b[MAXP + 1];
   u64 taupre[MAXP + 1];       // sum of tau_q over q < p
@@ -65,6 +61,13 @@ struct FShared {
   int red32[32];
   int ent[MAXP + 1];          // class boundaries in key order
   int n_phases, seg_end, fallback;
+  // two-tile ring of difference arrays: constant terms and slopes.  Round e of the ring (0 <= e <
+  // 2*TILE) lives at word e + 4*(e/32): four spare words after every 32 keep the 16-byte loads of
+  // the scan (a thread owns ITEMS consecutive rounds) free of bank conflicts while the index of an
+  // event stays a shift and an add.  Last in the struct: the kernel for evaluations that walk no
+  // rounds is launched without this part.
+  alignas(16) u32 dA[RINGW];
+  alignas(16) u32 dB[RINGW];
 };
 
 // floor(r * tau / k) for r, tau, k below 2^31 with a result below 2^31
@@ -678,7 +681,11 @@ struct FAcc {
   i64 peak64 = 0;
 };
 
-__global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_eval(BuildParams p) {
+// LIGHT: the variant for evaluations that walk no rounds (schedule only, or SPS / SimS whose peak
+// comes from the run ends): no ring in shared memory and fewer registers, so that three CTAs fit an
+// SM; an evaluation that needs its rounds walked is passed on to the full variant through a list.
+template <bool LIGHT>
+__global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 1 : KVS_EVAL_MIN_CTAS) k_fused_eval(BuildParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   FShared& sh = *reinterpret_cast<FShared*>(smem_raw);
   const int tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
@@ -689,7 +696,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
   uint2* const list0 = reinterpret_cast<uint2*>(reinterpret_cast<unsigned char*>(G) + ((static_cast<size_t>(p.max_jobs) / SEG + 2) * MAXP * 4));
   uint2* const list1 = list0 + (p.max_jobs + 1);
   u32* const fin_start = reinterpret_cast<u32*>(p.fin_rank) + static_cast<i64>(blockIdx.x) * p.max_jobs;
-  {
+  if (!LIGHT) {
     for (int i = tid; i < RINGW; i += T) { sh.dA[i] = 0; sh.dB[i] = 0; }
   }
 
@@ -701,8 +708,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
       sh.n_runs = 0;
     }
     __syncthreads();
-    const i64 e = sh.next_eval;
-    if (e >= p.P) break;
+    const i64 slot_no = sh.next_eval;
+    if (slot_no >= (p.eval_list ? static_cast<i64>(*p.eval_count) : p.P)) break;
+    const i64 e = p.eval_list ? p.eval_list[slot_no] : slot_no;
     const kvs_setting st = p.settings[e];
     const i64 lo = p.job_off[st.instance];
     const InstStats stats = p.stats[st.instance];
@@ -734,6 +742,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
     const bool want32 = p.out.job_start || p.out.job_completion;
     const bool event_form = p.do_profile && !geometric && p.prefix_s != nullptr && prof_cap == 0;
     const bool walk = p.do_profile && !event_form;            // rounds are walked tile by tile
+    if (LIGHT && walk) {
+      if (tid == 0) p.walk_list[atomicAdd(p.walk_count, 1ull)] = e;
+      continue;
+    }
 
     int status = stats.flags;
     if (!status && (X < 1 || stats.o_max > X)) status = KVS_EVAL_INFEASIBLE;
@@ -1104,7 +1116,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
           }
           __syncthreads();     // Z is scratch of the next window too
         }
-      } else if (walk) {
+      } else if (!LIGHT && walk) {
         bool list_mode = false;
         uint2* cur = list0;
         uint2* nxt = list1;
@@ -1265,22 +1277,30 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_fused_e
 
 }  // namespace
 
-static size_t fused_smem_bytes() { return sizeof(FShared); }
+static size_t fused_smem_bytes(bool light) { return light ? offsetof(FShared, dA) : sizeof(FShared); }
 
-int kvs_fused_ctas_per_sm() {
+template <bool LIGHT>
+static int ctas_per_sm() {
   int n = 0;
-  cudaFuncSetAttribute(k_fused_eval, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes()));
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_fused_eval, KVS_EVAL_THREADS, fused_smem_bytes()) != cudaSuccess) n = 1;
+  cudaFuncSetAttribute(k_fused_eval<LIGHT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(LIGHT)));
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_fused_eval<LIGHT>, KVS_EVAL_THREADS, fused_smem_bytes(LIGHT)) != cudaSuccess) n = 1;
   return n < 1 ? 1 : n;
 }
 
-cudaError_t kvs_launch_fused(const BuildParams& p, int grid, cudaStream_t stream) {
+int kvs_fused_ctas_per_sm(int light) { return light ? ctas_per_sm<true>() : ctas_per_sm<false>(); }
+
+// The caller zeroes the counters.  light: the variant without the ring (see k_fused_eval).
+cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, cudaStream_t stream) {
   if (p.P <= 0) return cudaSuccess;
-  cudaError_t err = cudaFuncSetAttribute(k_fused_eval, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(fused_smem_bytes()));
-  if (err != cudaSuccess) return err;
-  err = cudaMemsetAsync(p.counter, 0, 16, stream);   // work counter and length of the list of left-over evaluations
-  if (err != cudaSuccess) return err;
-  k_fused_eval<<<grid, KVS_EVAL_THREADS, fused_smem_bytes(), stream>>>(p);
+  cudaError_t err;
+  if (light) {
+    err = cudaFuncSetAttribute(k_fused_eval<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(true)));
+    if (err != cudaSuccess) return err;
+    k_fused_eval<true><<<grid, KVS_EVAL_THREADS, fused_smem_bytes(true), stream>>>(p);
+  } else {
+    err = cudaFuncSetAttribute(k_fused_eval<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(false)));
+    if (err != cudaSuccess) return err;
+    k_fused_eval<false><<<grid, KVS_EVAL_THREADS, fused_smem_bytes(false), stream>>>(p);
+  }
   return cudaGetLastError();
 }

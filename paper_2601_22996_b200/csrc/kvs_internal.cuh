@@ -69,9 +69,12 @@ struct BuildParams {
   // The 32-bit fast kernel appends the evaluations it leaves to the general kernel here ...
   i64* slow_list;
   ull* slow_count;
-  // ... and the general kernel, when given a list, works through eval_list[0 .. *eval_count)
+  // ... and a kernel that is given a list works through eval_list[0 .. *eval_count)
   const i64* eval_list;
   const ull* eval_count;
+  // evaluations the light variant of the fast kernel passes on to the full one
+  i64* walk_list;
+  ull* walk_count;
 };
 
 struct SortParams {
@@ -119,8 +122,8 @@ struct SweepParams {
 cudaError_t kvs_launch_sort(const SortParams& p, int grid, cudaStream_t stream);
 cudaError_t kvs_launch_build(const BuildParams& p, int grid, cudaStream_t stream);
 int kvs_build_ctas_per_sm();
-cudaError_t kvs_launch_fused(const BuildParams& p, int grid, cudaStream_t stream);
-int kvs_fused_ctas_per_sm();
+cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, cudaStream_t stream);
+int kvs_fused_ctas_per_sm(int light);
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_bounds(const i64* job_off, const int32_t* o, const InstStats* stats, const kvs_setting* settings,
                               i64 P, const kvs_bounds_out& out, int grid, cudaStream_t stream);
