@@ -25,11 +25,12 @@ sys.path.insert(0, ROOT)
 from paper_2601_22996_b200 import workloads  # noqa: E402
 
 METRIC, UNIT = "schedule_evaluation_job_steps_per_sec", "job-steps/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_fused_eval launch, from the ncu capture summarised in
-# profiles/k_fused_eval_c5.md (592 instances of config 5, all four families: 2,368 evaluations, 4.685 GB).
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, the full variant of
+# k_fused_eval (it takes the geometric evaluations), from the ncu capture summarised in
+# profiles/k_fused_eval_c5.md (592 instances of config 5: 1,184 GBA/GSA evaluations, 3.555 GB).
 # Traffic grows with the number of evaluations (each CTA works on one at a time), so a launch is scaled
 # by its evaluation count.  Valid for the kernel state named in that file; set to None when the kernel changes.
-C5_TRAFFIC_BYTES_PER_EVALUATION = 4.684714e9 / 2368
+C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION = 3.555471e9 / 1184
 WORKLOADS = {
     # name: (generator, instances, jobs per instance, families, description)
     "c2": ("config2", 1024, 10_000, ["GBA", "GSA"], "config 2: 1,024 instances x 10,000 jobs, M in {2^17..2^24}, GBA+GSA"),
@@ -240,12 +241,15 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     ms = e0.elapsed_time(e1)
     # kernel durations (CUDA events recorded by the library on its stream around each kernel)
-    sort_ms, build_ms = [], []
+    sort_ms, build_ms, light_ms, full_ms = [], [], [], []
     for _ in range(args.steps):
         step()
         a, b = ctx.last_timing()
+        _, c, d = ctx.last_timing_split()
         sort_ms.append(a)
         build_ms.append(b)
+        light_ms.append(c)
+        full_ms.append(d)
     ctx.set_timing(False)
     assert int((ev["status"] != 0).sum()) == 0, "an evaluation reported a non-zero status"
     job_steps = int(ev["job_steps"].sum())
@@ -271,7 +275,8 @@ def run_ours(args):
         e2e = (e2e_s, h2d, d2h)
 
     # max over ranks, totals over ranks
-    stats = torch.tensor([ms, e2e[0] if e2e else 0.0, float(np.mean(build_ms)), float(np.mean(sort_ms))], dtype=torch.float64, device=dev)
+    stats = torch.tensor([ms, e2e[0] if e2e else 0.0, float(np.mean(build_ms)), float(np.mean(sort_ms)),
+                          float(np.mean(light_ms)), float(np.mean(full_ms))], dtype=torch.float64, device=dev)
     tot = torch.tensor([float(job_steps), float(P)], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(stats, op=dist.ReduceOp.MAX)
@@ -280,18 +285,22 @@ def run_ours(args):
         if world > 1:
             dist.destroy_process_group()
         return
-    ms, e2e_s, build_avg, sort_avg = [float(x) for x in stats.tolist()]
+    ms, e2e_s, build_avg, sort_avg, light_avg, full_avg = [float(x) for x in stats.tolist()]
     steps_all, evals_all = tot.tolist()
     sec_per_step = ms / 1e3 / args.steps
     share = len(fams) * (len(inst.meta["M"]) if "M" in inst.meta and name == "c2" else 1)
-    # algorithmic bytes of one builder/evaluator launch on this rank: inputs once per instance,
-    # start + completion per job and evaluation, one int32 per profile round, scalars
-    alg_bytes = 8 * N + 8 * P * n + 4 * rounds + 57 * P
+    # Dominant kernel: the full variant of k_fused_eval, which takes the geometric (GBA/GSA) evaluations.
+    # Its algorithmic bytes on this rank: the instances once, start + completion per job and evaluation,
+    # one int32 per profile round, scalars.  (The light variant does the same for SPS / SimS without
+    # profile rounds; `stage_algorithmic_bytes` is the figure for both together.)
+    geo = int((settings["family"] <= 1).sum())
+    alg_bytes = (8 * N if geo else 0) + 8 * geo * n + 4 * rounds + 57 * geo
+    stage_bytes = 8 * N + 8 * P * n + 4 * rounds + 57 * P
     peak_gbs, peak_kind = load_peaks()
-    achieved = alg_bytes / (build_avg * 1e-3) / 1e9
+    achieved = alg_bytes / (full_avg * 1e-3) / 1e9 if geo else 0.0
     traffic = None
-    if name == "c5" and len(fams) == 4 and C5_TRAFFIC_BYTES_PER_EVALUATION:
-        traffic = C5_TRAFFIC_BYTES_PER_EVALUATION * P
+    if name == "c5" and geo and C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION:
+        traffic = C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION * geo
     line = {
         "metric": METRIC, "value": steps_all / sec_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * sec_per_step, "higher_is_better": True, "scaling": "weak",
@@ -300,10 +309,12 @@ def run_ours(args):
                    "evaluations_per_gpu": P, "evaluations_sharing_an_instance": share, "alpha": "2/1",
                    "profile_rounds_per_gpu": rounds, "l2": "inputs and outputs larger than L2"},
         "evaluations_per_sec": evals_all / sec_per_step,
-        "kernels_ms": {"k_stats_sort": sort_avg, "k_fused_eval+k_build_eval": build_avg},
+        "kernels_ms": {"k_stats_sort": sort_avg, "k_fused_eval<light>": light_avg, "k_fused_eval<full>+k_build_eval": full_avg,
+                       "builder_evaluator_stage": build_avg},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
-                     "traffic": traffic, "peak_kind": peak_kind, "kernel": "k_fused_eval", "algorithmic_bytes": alg_bytes},
-        "gpu_launches": 3 * args.steps, "clocks": clocks,
+                     "traffic": traffic, "peak_kind": peak_kind, "kernel": "k_fused_eval<full>", "algorithmic_bytes": alg_bytes,
+                     "stage_algorithmic_bytes": stage_bytes, "stage_frac": stage_bytes / (build_avg * 1e-3) / 1e9 / peak_gbs},
+        "gpu_launches": 4 * args.steps, "clocks": clocks,
     }
     if e2e:
         line["e2e"] = {"value": steps_all / (e2e_s / args.steps), "unit": UNIT, "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2]}

@@ -77,6 +77,10 @@ const char* kvs_last_error(const kvs_ctx* ctx);
  * the most recent fused call (0 if timing was off). */
 int kvs_set_timing(kvs_ctx* ctx, int32_t enabled);
 int kvs_last_timing(kvs_ctx* ctx, float* sort_ms, float* build_ms);
+/* The same with the builder/evaluator stage split: the variant of the fast kernel for evaluations
+ * that walk no rounds (`light_ms`) and everything after it - the full variant and the general
+ * kernel (`full_ms`).  A call that took the general kernel alone reports it all as `full_ms`. */
+int kvs_last_timing_split(kvs_ctx* ctx, float* sort_ms, float* light_ms, float* full_ms);
 
 /* Workspace needed by any call whose sizes do not exceed the given ones.
  *   n_jobs_total           sum of jobs over all instances of a call

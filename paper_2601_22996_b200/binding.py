@@ -74,7 +74,7 @@ class _BoundsOut(Structure):
     _fields_ = [("upper_gba", c_void_p), ("upper_gsa", c_void_p), ("lower_2m", c_void_p), ("status", c_void_p)]
 
 
-EXPORTS = ["kvs_init", "kvs_destroy", "kvs_last_error", "kvs_set_timing", "kvs_last_timing", "kvs_workspace_bytes",
+EXPORTS = ["kvs_init", "kvs_destroy", "kvs_last_error", "kvs_set_timing", "kvs_last_timing", "kvs_last_timing_split", "kvs_workspace_bytes",
            "kvs_build_schedule", "kvs_evaluate_built", "kvs_evaluate_built_host", "kvs_evaluate_schedule", "kvs_sweep",
            "kvs_evaluate_schedule_noalloc", "kvs_bounds"]
 
@@ -96,6 +96,7 @@ def load(path: str | None = None):
         L.kvs_last_error.restype = c_char_p
         L.kvs_set_timing.argtypes = [c_void_p, c_int32]
         L.kvs_last_timing.argtypes = [c_void_p, POINTER(c_float), POINTER(c_float)]
+        L.kvs_last_timing_split.argtypes = [c_void_p, POINTER(c_float), POINTER(c_float), POINTER(c_float)]
         L.kvs_workspace_bytes.argtypes = [c_int64, c_int64, c_int64, c_int64, c_int64, c_int32, POINTER(c_uint64)]
         L.kvs_build_schedule.argtypes = [c_void_p, POINTER(_Instances), c_void_p, c_int64, POINTER(_ScheduleOut), POINTER(_EvalOut)]
         L.kvs_evaluate_built.argtypes = L.kvs_build_schedule.argtypes
@@ -210,6 +211,12 @@ class Context:
         a, b = c_float(0), c_float(0)
         self._check(self._lib.kvs_last_timing(self._ctx, ctypes.byref(a), ctypes.byref(b)))
         return float(a.value), float(b.value)
+
+    def last_timing_split(self) -> tuple[float, float, float]:
+        """Device milliseconds of the ordering kernel, the light variant and the full variant (+ general kernel)."""
+        a, b, c = c_float(0), c_float(0), c_float(0)
+        self._check(self._lib.kvs_last_timing_split(self._ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
+        return float(a.value), float(b.value), float(c.value)
 
     @staticmethod
     def _instances(inst: Instances, window: int = 0, max_jobs: int | None = None):

@@ -22,7 +22,8 @@ struct kvs_ctx {
   int light_ctas_per_sm = 1;
   bool timing = false;
   bool timed = false;
-  cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before the ordering kernel, between, after the builder
+  bool split_timed = false;   // the last timed call took the fast path (event between its two variants)
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};   // before the ordering kernel, after it, after the last kernel, after the light variant
   // host entry point: input copies run on a stream of their own, one event per chunk of instances
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t chunk_ev[KVS_HOST_CHUNKS + 1] = {};
@@ -280,6 +281,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
       ce = kvs_launch_fused(bp, grid_for(ctx->light_ctas_per_sm), 1, ctx->stream);
       if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
     }
+    if (ctx->timing && !rg) cudaEventRecord(ctx->ev[3], ctx->stream);
     bp.counter = counters + 4;
     bp.eval_list = bp.walk_list;
     bp.eval_count = bp.walk_count;
@@ -291,7 +293,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.counter = counters + 2;
   ce = kvs_launch_build(bp, grid_for(ctx->build_ctas_per_sm), ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "build launch");
-  if (ctx->timing && !rg) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; }
+  if (ctx->timing && !rg) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; ctx->split_timed = fast; }
   return KVS_OK;
 }
 
@@ -359,6 +361,25 @@ int kvs_last_timing(kvs_ctx* ctx, float* sort_ms, float* build_ms) {
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaEventSynchronize");
   if (sort_ms) cudaEventElapsedTime(sort_ms, ctx->ev[0], ctx->ev[1]);
   if (build_ms) cudaEventElapsedTime(build_ms, ctx->ev[1], ctx->ev[2]);
+  return KVS_OK;
+}
+
+int kvs_last_timing_split(kvs_ctx* ctx, float* sort_ms, float* light_ms, float* full_ms) {
+  if (!ctx) return KVS_E_STATE;
+  if (sort_ms) *sort_ms = 0.f;
+  if (light_ms) *light_ms = 0.f;
+  if (full_ms) *full_ms = 0.f;
+  if (!ctx->timed) return KVS_OK;
+  cudaError_t ce = cudaEventSynchronize(ctx->ev[2]);
+  if (ce != cudaSuccess) return fail_cuda(ctx, ce, "cudaEventSynchronize");
+  if (sort_ms) cudaEventElapsedTime(sort_ms, ctx->ev[0], ctx->ev[1]);
+  // the event between the two variants exists only on the fast path
+  if (cudaEventQuery(ctx->ev[3]) == cudaSuccess && ctx->split_timed) {
+    if (light_ms) cudaEventElapsedTime(light_ms, ctx->ev[1], ctx->ev[3]);
+    if (full_ms) cudaEventElapsedTime(full_ms, ctx->ev[3], ctx->ev[2]);
+  } else if (full_ms) {
+    cudaEventElapsedTime(full_ms, ctx->ev[1], ctx->ev[2]);
+  }
   return KVS_OK;
 }
 
