@@ -647,8 +647,8 @@ __device__ __forceinline__ void scan_tile(FShared& sh, int buf, i64 t0, int wlen
       int4* dst = reinterpret_cast<int4*>(prof + t0 + e0);
 #pragma unroll
       for (int v = 0; v < VEC; ++v)
-        dst[v] = make_int4(static_cast<int>(mem[4 * v]), static_cast<int>(mem[4 * v + 1]),
-                           static_cast<int>(mem[4 * v + 2]), static_cast<int>(mem[4 * v + 3]));
+        __stcs(&dst[v], make_int4(static_cast<int>(mem[4 * v]), static_cast<int>(mem[4 * v + 1]),
+                                  static_cast<int>(mem[4 * v + 2]), static_cast<int>(mem[4 * v + 3])));   // written once, never re-read: streaming
     }
     return;
   }
@@ -944,8 +944,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             } else {
               ++acc.unfinished;
             }
-            if (out_start) out_start[j] = start;
-            if (out_done) out_done[j] = done;
+            if (out_start) __stcs(&out_start[j], start);
+            if (out_done) __stcs(&out_done[j], done);
           }
         }
       } else {
@@ -999,8 +999,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
               const u32 done = stt + ov;
               acc.hmax = max(acc.hmax, done);
               acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
-              if (out_start) out_start[j] = static_cast<int32_t>(stt);
-              if (out_done) out_done[j] = static_cast<int32_t>(done);
+              if (out_start) __stcs(&out_start[j], static_cast<int32_t>(stt));
+              if (out_done) __stcs(&out_done[j], static_cast<int32_t>(done));
             }
           }
         }
@@ -1013,8 +1013,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             const u32 done = stt + oj;
             acc.hmax = max(acc.hmax, done);
             acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
-            if (out_start) out_start[j] = static_cast<int32_t>(stt);
-            if (out_done) out_done[j] = static_cast<int32_t>(done);
+            if (out_start) __stcs(&out_start[j], static_cast<int32_t>(stt));
+            if (out_done) __stcs(&out_done[j], static_cast<int32_t>(done));
           }
         }
       }

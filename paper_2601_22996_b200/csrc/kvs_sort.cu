@@ -142,9 +142,9 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       __syncthreads();
       for (int j = seg_lo + tid; j < seg_hi; j += T) {
         const int idx = p.perm[lo + j];
-        p.sorted_s[lo + j] = p.s[lo + idx];
-        p.sorted_o[lo + j] = p.o[lo + idx];
-        if (p.key) p.sorted_key[lo + j] = p.key[lo + idx];
+        __stcs(&p.sorted_s[lo + j], p.s[lo + idx]);     // streaming stores: read back much later, by another kernel
+        __stcs(&p.sorted_o[lo + j], p.o[lo + idx]);
+        if (p.key) __stcs(&p.sorted_key[lo + j], p.key[lo + idx]);
         if (p.iperm) p.iperm[lo + idx] = j;
       }
       __syncthreads();
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
           if (static_cast<int>(lane_id()) >= d) wi += y;
         }
         const i64 before = run + __shfl_sync(0xffffffffu, wi - w, tid >> 5);   // all lanes take part in the shuffle
-        if (j < n) ps[j + 1] = before + incl;
+        if (j < n) __stcs(&ps[j + 1], before + incl);
         run += __shfl_sync(0xffffffffu, wi, 31);
       }
     }
