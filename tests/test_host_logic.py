@@ -90,3 +90,19 @@ def test_two_rank_reporting_over_gloo():
         assert times == [11.0, 5.0] and counts == [float(total), 4.0]     # max over ranks, sum over ranks
     whole = workloads.config2(n_inst=4, n=100)
     assert int(whole.o.sum()) == total                                    # the two shards are the 4-instance stream
+
+
+def test_reference_arm_prints_one_json_line():
+    """bench.py --impl reference times the oracle on the host and prints the contract's JSON line."""
+    import json
+    import subprocess
+    import sys
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0",
+                          "--cpu-seconds", "0.5"], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["value"] > 0 and d["unit"] == "job-steps/s" and d["higher_is_better"] is True
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
