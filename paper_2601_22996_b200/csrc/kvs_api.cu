@@ -265,6 +265,13 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
       if (do_profile && settings[e].family <= KVS_GSA) ids[static_cast<size_t>(n_full++)] = e;
     for (int64_t e = 0; e < P; ++e)
       if (!(do_profile && settings[e].family <= KVS_GSA)) ids[static_cast<size_t>(n_full + n_light++)] = e;
+    // Longest first: the rounds of a schedule grow as the budget shrinks and the slicing algorithm
+    // visits more runs than the batching one, and the CTAs draw evaluations in list order, so this
+    // order keeps the last CTAs from finishing a long evaluation alone.
+    std::stable_sort(ids.begin(), ids.begin() + n_full, [&](int64_t a, int64_t b) {
+      if (settings[a].M != settings[b].M) return settings[a].M < settings[b].M;
+      return settings[a].family > settings[b].family;
+    });
     const unsigned long long init[8] = {0, 0, 0, static_cast<unsigned long long>(n_full), 0, static_cast<unsigned long long>(n_light), 0, 0};
     if ((ce = cudaMemcpyAsync(counters, init, sizeof(init), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
         (n_full && (ce = cudaMemcpyAsync(ws + L.walk_list, ids.data(), static_cast<size_t>(n_full) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) ||
