@@ -30,7 +30,7 @@ METRIC, UNIT = "schedule_evaluation_job_steps_per_sec", "job-steps/s"
 # profiles/k_fused_eval_c5.md (592 instances of config 5: 1,184 GBA/GSA evaluations, 3.374 GB).
 # Traffic grows with the number of evaluations (each CTA works on one at a time), so a launch is scaled
 # by its evaluation count.  Valid for the kernel state named in that file; set to None when the kernel changes.
-C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION = 3.374415e9 / 1184
+C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION = 3.366606e9 / 1184
 WORKLOADS = {
     # name: (generator, instances, jobs per instance, families, description)
     "c2": ("config2", 1024, 10_000, ["GBA", "GSA"], "config 2: 1,024 instances x 10,000 jobs, M in {2^17..2^24}, GBA+GSA"),
