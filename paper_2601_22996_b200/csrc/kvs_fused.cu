@@ -332,6 +332,113 @@ __device__ __forceinline__ void visit_runs(FShared& sh, const PhaseView& P, int 
   }
 }
 
+// The run visit of a phase with carried jobs in which at least eight runs start per round (and the
+// slice is shorter than a tile).  A lane's up to eight participants then start in one round or in
+// two consecutive ones, so the lane first treats all of them as killed at the end of their slot:
+// one start event and one end event per round, from sums over its participants, without a loop
+// over runs.  Afterwards each participant that completes before the end of its slot moves its own
+// end event from start + tau to start + o.  Same events in total as visit_runs<false, true>.
+__device__ __forceinline__ void visit_runs_sliced(FShared& sh, const PhaseView& P, int ra, int rb, int trel, int buf, u64 kinv) {
+  if (ra >= rb) return;
+  u32* const dA = sh.dA;
+  u32* const dB = sh.dB;
+  const u32 tau = P.tau, k = P.k;
+  const int warp = threadIdx.x >> 5;
+  const bool vec = (reinterpret_cast<uintptr_t>(P.S) & 15u) == 0;
+  int seg_a, seg_b;
+  segment_range<true>(P, ra, rb, &seg_a, &seg_b);
+  for (int seg = seg_a + warp; seg < seg_b; seg += WARPS) {
+    const int xb0 = seg * SEG + 8 * static_cast<int>(lane_id());
+    const bool vload = vec && xb0 + 8 <= P.n_src;
+    uint4 a0 = make_uint4(0, 0, 0, 0), a1 = a0;
+    if (vload) {
+      a0 = __ldg(reinterpret_cast<const uint4*>(P.S + xb0));
+      a1 = __ldg(reinterpret_cast<const uint4*>(P.S + xb0) + 1);
+    }
+    const LaneGroup g = lane_group<true>(P, seg);
+    const int cnt = __popc(g.bits);
+    const int skip = max(0, ra - g.r_first);
+    const int take = min(cnt, rb - g.r_first) - skip;
+    if (__ballot_sync(0xffffffffu, take > 0) == 0) continue;
+    if (take <= 0) continue;
+    // the lane's participants with ranks inside [ra, rb)
+    u32 bits = g.bits;
+    for (int i = 0; i < skip; ++i) bits &= bits - 1u;
+    for (int extra = __popc(bits) - take; extra > 0; --extra) bits &= ~(0x80000000u >> __clz(bits));
+    u32 s_[8];
+    if (vload) {
+      s_[0] = a0.x; s_[1] = a0.y; s_[2] = a0.z; s_[3] = a0.w; s_[4] = a1.x; s_[5] = a1.y; s_[6] = a1.z; s_[7] = a1.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s_[j] = (bits >> j & 1u) ? static_cast<u32>(__ldg(P.S + g.xb + j)) : 0u;
+    }
+    const u32 n = static_cast<u32>(take);
+    const u32 r0 = static_cast<u32>(g.r_first + skip);
+    const u32 q0 = slot_mul(r0, tau, k, kinv);
+    // rank r0 + j starts in round q0 + floor((rem + j tau) / k): the first m stay in round q0
+    const u32 rem = static_cast<u32>(static_cast<u64>(r0) * tau - static_cast<u64>(q0) * k);
+    u32 m = 1;
+#pragma unroll
+    for (u32 j = 1; j < 8; ++j) m += (rem + j * tau < k) ? 1u : 0u;
+    m = min(m, n);
+    u32 sumA = 0, sumB = 0, idx = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (bits >> j & 1u) {
+        const u32 v = s_[j] + 1u;
+        if (idx < m) sumA += v; else sumB += v;
+        ++idx;
+      }
+    }
+    const int srel = static_cast<int>(q0) - trel;
+    {
+      const u32 c = sumA - m * (P.base + q0);
+      const int si = ring(buf, srel);
+      atomicAdd(&dA[si], c);
+      atomicAdd(&dB[si], m);
+      if (q0 + tau < P.len) {
+        const int ei = ring(buf, srel + static_cast<int>(tau));
+        atomicAdd(&dA[ei], 0u - c);
+        atomicAdd(&dB[ei], 0u - m);
+      }
+    }
+    if (n > m) {
+      const u32 c = sumB - (n - m) * (P.base + q0 + 1u);
+      const int si = ring(buf, srel + 1);
+      atomicAdd(&dA[si], c);
+      atomicAdd(&dB[si], n - m);
+      if (q0 + 1u + tau < P.len) {
+        const int ei = ring(buf, srel + 1 + static_cast<int>(tau));
+        atomicAdd(&dA[ei], 0u - c);
+        atomicAdd(&dB[ei], 0u - (n - m));
+      }
+    }
+    // completing jobs: the end moves from start + tau to start + o
+    u32 fb = g.fbits & bits;
+    while (fb) {
+      const int j = __ffs(static_cast<int>(fb)) - 1;
+      fb &= fb - 1u;
+      const u32 oi = static_cast<u32>(__ldg(P.O + g.xb + j));
+      if (oi < tau) {
+        const u32 before = static_cast<u32>(__popc(bits & ((1u << j) - 1u)));
+        const u32 q = q0 + (before >= m ? 1u : 0u);
+        const u32 c = static_cast<u32>(__ldg(P.S + g.xb + j)) + 1u - P.base - q;
+        const int sr = static_cast<int>(q) - trel;
+        if (q + oi < P.len) {
+          const int ei = ring(buf, sr + static_cast<int>(oi));
+          atomicAdd(&dA[ei], 0u - c);
+          atomicAdd(&dB[ei], 0xffffffffu);
+        }
+        if (q + tau < P.len) {
+          const int ki = ring(buf, sr + static_cast<int>(tau));
+          atomicAdd(&dA[ki], c);
+          atomicAdd(&dB[ki], 1u);
+        }
+      }
+    }
+  }
+}
+
 // Exclusive block scan of a small per-thread count; returns this thread's offset, total in *total.
 __device__ __forceinline__ int block_count_scan(int v, int* red32, int* total) {
   int incl = v;
@@ -1221,6 +1328,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             if (ph < n_pure) pure_phase_events(sh, P, PS, N, u0, buf);
             else if (sim) visit_runs<true, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             else if (list_mode) C_next = visit_list(sh, P, V, nxt, C_next, r_next, r_b, u0, buf, dense);
+            else if (carry && P.tau < static_cast<u32>(TILE) && P.k >= 8u * P.tau) visit_runs_sliced(sh, P, r_next, r_b, u0, buf, sh.kinv[ph]);
             else if (carry) visit_runs<false, true>(sh, P, r_next, r_b, u0, buf, dense, combine);
             else visit_runs<false, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             r_next = r_b;
