@@ -21,8 +21,11 @@ __device__ __forceinline__ int32_t key_at(const SortParams& p, i64 lo, int idx) 
   return p.key ? p.key[lo + idx] : p.o[lo + idx];
 }
 
-// Sort positions [seg_lo, seg_hi) of the instance starting at global job index lo.
-__device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
+// Sort positions [seg_lo, seg_hi) of the instance starting at global job index lo.  The last pass
+// holds every job's key when it places the job, so it also writes the keys in sorted order (one more
+// scattered store that merges in L2 like the index, instead of a gather afterwards); returns
+// whether it did.
+__device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
                              u32 (*warp_cnt)[256], u32* bucket, u32 (*hist)[256]) {
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n = seg_hi - seg_lo;
@@ -30,7 +33,7 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
   if (passes == 0 || n <= 1) {
     for (int j = tid; j < n; j += T) out[j] = seg_lo + j;
     __syncthreads();
-    return;
+    return false;
   }
   // digit histograms of all passes in one sweep
   for (int i = tid; i < 4 * 256; i += T) (&hist[0][0])[i] = 0;
@@ -59,6 +62,7 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
     const bool to_perm = ((passes - 1 - pass) & 1) == 0;
     int32_t* dst = (to_perm ? p.perm : p.perm_tmp) + lo + seg_lo;
     const int32_t* src = (to_perm ? p.perm_tmp : p.perm) + lo + seg_lo;
+    int32_t* const key_dst = pass == passes - 1 ? (p.key ? p.sorted_key : p.sorted_o) + lo + seg_lo : nullptr;
     if (tid < 256) bucket[tid] = hist[pass][tid];
     for (int j0 = 0; j0 < n; j0 += T) {
       for (int i = tid; i < WARPS * 256; i += T) (&warp_cnt[0][0])[i] = 0;
@@ -66,10 +70,11 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
       const int j = j0 + tid;
       const bool valid = j < n;
       int idx = 0;
-      u32 digit = 256;  // sentinel for lanes past the end
+      u32 key = 0, digit = 256;  // sentinel for lanes past the end
       if (valid) {
         idx = pass == 0 ? seg_lo + j : src[j];
-        digit = (static_cast<u32>(key_at(p, lo, idx)) >> (8 * pass)) & 255u;
+        key = static_cast<u32>(key_at(p, lo, idx));
+        digit = (key >> (8 * pass)) & 255u;
       }
       const u32 peers = __match_any_sync(0xffffffffu, digit);
       const u32 rank = __popc(peers & lanemask_lt());
@@ -85,10 +90,15 @@ __device__ void sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
         bucket[tid] = acc;
       }
       __syncthreads();
-      if (valid) dst[warp_cnt[warp][digit] + rank] = idx;
+      if (valid) {
+        const u32 pos = warp_cnt[warp][digit] + rank;
+        dst[pos] = idx;
+        if (key_dst) key_dst[pos] = static_cast<int32_t>(key);
+      }
       __syncthreads();
     }
   }
+  return true;
 }
 
 __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
@@ -138,13 +148,17 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       }
       __syncthreads();
       const int seg_hi = seg_end;
-      sort_segment(p, lo, seg_lo, seg_hi, passes, warp_cnt, bucket, hist);
+      const bool have_key = sort_segment(p, lo, seg_lo, seg_hi, passes, warp_cnt, bucket, hist);
       __syncthreads();
       for (int j = seg_lo + tid; j < seg_hi; j += T) {
         const int idx = p.perm[lo + j];
         __stcs(&p.sorted_s[lo + j], p.s[lo + idx]);     // streaming stores: read back much later, by another kernel
-        __stcs(&p.sorted_o[lo + j], p.o[lo + idx]);
-        if (p.key) __stcs(&p.sorted_key[lo + j], p.key[lo + idx]);
+        if (p.key) {
+          __stcs(&p.sorted_o[lo + j], p.o[lo + idx]);
+          if (!have_key) __stcs(&p.sorted_key[lo + j], p.key[lo + idx]);
+        } else if (!have_key) {
+          __stcs(&p.sorted_o[lo + j], p.o[lo + idx]);
+        }
         if (p.iperm) p.iperm[lo + idx] = j;
       }
       __syncthreads();
