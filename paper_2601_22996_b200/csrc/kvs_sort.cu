@@ -25,7 +25,9 @@ __device__ __forceinline__ int32_t key_at(const SortParams& p, i64 lo, int idx) 
 // holds every job's key when it places the job, so it also writes the keys in sorted order (one more
 // scattered store that merges in L2 like the index, instead of a gather afterwards); returns
 // whether it did.
-__device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes,
+// packed: indices and keys are below 2^16, so a pass that is not the last stores (key << 16 | index)
+// and the next pass needs no look-up of the key through the index.
+__device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes, bool packed,
                              u32 (*warp_cnt)[256], u32* bucket, u32 (*hist)[256]) {
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n = seg_hi - seg_lo;
@@ -72,8 +74,9 @@ __device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
       int idx = 0;
       u32 key = 0, digit = 256;  // sentinel for lanes past the end
       if (valid) {
-        idx = pass == 0 ? seg_lo + j : src[j];
-        key = static_cast<u32>(key_at(p, lo, idx));
+        if (pass == 0) { idx = seg_lo + j; key = static_cast<u32>(key_at(p, lo, idx)); }
+        else if (packed) { const u32 rec = static_cast<u32>(src[j]); idx = static_cast<int>(rec & 0xffffu); key = rec >> 16; }
+        else { idx = src[j]; key = static_cast<u32>(key_at(p, lo, idx)); }
         digit = (key >> (8 * pass)) & 255u;
       }
       const u32 peers = __match_any_sync(0xffffffffu, digit);
@@ -92,7 +95,7 @@ __device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
       __syncthreads();
       if (valid) {
         const u32 pos = warp_cnt[warp][digit] + rank;
-        dst[pos] = idx;
+        dst[pos] = (packed && !key_dst) ? static_cast<int32_t>(key << 16 | static_cast<u32>(idx)) : idx;
         if (key_dst) key_dst[pos] = static_cast<int32_t>(key);
       }
       __syncthreads();
@@ -148,7 +151,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       }
       __syncthreads();
       const int seg_hi = seg_end;
-      const bool have_key = sort_segment(p, lo, seg_lo, seg_hi, passes, warp_cnt, bucket, hist);
+      const bool have_key = sort_segment(p, lo, seg_lo, seg_hi, passes, n <= 65536 && key_max < 65536, warp_cnt, bucket, hist);
       __syncthreads();
       for (int j = seg_lo + tid; j < seg_hi; j += T) {
         const int idx = p.perm[lo + j];
