@@ -28,7 +28,7 @@ __device__ __forceinline__ int32_t key_at(const SortParams& p, i64 lo, int idx) 
 // packed: indices and keys are below 2^16, so a pass that is not the last stores (key << 16 | index)
 // and the next pass needs no look-up of the key through the index.
 __device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi, int passes, bool packed,
-                             u32 (*warp_cnt)[256], u32* bucket, u32 (*hist)[256]) {
+                             u32 (*warp_cnt)[256], u32 (*warp_off)[256], u32 (*hist)[256]) {
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n = seg_hi - seg_lo;
   int32_t* const out = p.perm + lo + seg_lo;
@@ -39,6 +39,7 @@ __device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
   }
   // digit histograms of all passes in one sweep
   for (int i = tid; i < 4 * 256; i += T) (&hist[0][0])[i] = 0;
+  for (int i = tid; i < WARPS * 256; i += T) (&warp_cnt[0][0])[i] = 0;   // stays zero between tiles, see below
   __syncthreads();
   for (int j = tid; j < n; j += T) {
     u32 key = static_cast<u32>(key_at(p, lo, seg_lo + j));
@@ -65,10 +66,12 @@ __device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
     int32_t* dst = (to_perm ? p.perm : p.perm_tmp) + lo + seg_lo;
     const int32_t* src = (to_perm ? p.perm_tmp : p.perm) + lo + seg_lo;
     int32_t* const key_dst = pass == passes - 1 ? (p.key ? p.sorted_key : p.sorted_o) + lo + seg_lo : nullptr;
-    if (tid < 256) bucket[tid] = hist[pass][tid];
+    u32 bucket = tid < 256 ? hist[pass][tid] : 0u;   // thread d keeps the running position of digit d
     for (int j0 = 0; j0 < n; j0 += T) {
-      for (int i = tid; i < WARPS * 256; i += T) (&warp_cnt[0][0])[i] = 0;
-      __syncthreads();
+      // Two barriers per tile: the counts are written before the first and read before the second;
+      // the offsets are written between them and read after the second (and not overwritten
+      // before the first barrier of the next tile, which every thread reaches only after its store).
+      // The lane that wrote a count clears it after the second barrier.
       const int j = j0 + tid;
       const bool valid = j < n;
       int idx = 0;
@@ -81,33 +84,37 @@ __device__ bool sort_segment(const SortParams& p, i64 lo, int seg_lo, int seg_hi
       }
       const u32 peers = __match_any_sync(0xffffffffu, digit);
       const u32 rank = __popc(peers & lanemask_lt());
-      if (valid && rank == 0) warp_cnt[warp][digit] = __popc(peers);
+      const bool leader = valid && rank == 0;
+      if (leader) warp_cnt[warp][digit] = __popc(peers);
       __syncthreads();
       if (tid < 256) {
-        u32 acc = bucket[tid];
+        u32 acc = bucket;
+#pragma unroll
         for (int w = 0; w < WARPS; ++w) {
-          u32 t = warp_cnt[w][tid];
-          warp_cnt[w][tid] = acc;
-          acc += t;
+          warp_off[w][tid] = acc;
+          acc += warp_cnt[w][tid];
         }
-        bucket[tid] = acc;
+        bucket = acc;
       }
       __syncthreads();
       if (valid) {
-        const u32 pos = warp_cnt[warp][digit] + rank;
+        const u32 pos = warp_off[warp][digit] + rank;
         dst[pos] = (packed && !key_dst) ? static_cast<int32_t>(key << 16 | static_cast<u32>(idx)) : idx;
         if (key_dst) key_dst[pos] = static_cast<int32_t>(key);
       }
-      __syncthreads();
+      if (leader) warp_cnt[warp][digit] = 0;
+      __syncwarp();
     }
+    __syncthreads();   // the next pass reads what this one stored
   }
   return true;
 }
 
 __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
-  __shared__ u32 warp_cnt[WARPS][256];
+  extern __shared__ __align__(16) u32 dyn[];
+  u32 (*const warp_cnt)[256] = reinterpret_cast<u32 (*)[256]>(dyn);
+  u32 (*const warp_off)[256] = reinterpret_cast<u32 (*)[256]>(dyn + WARPS * 256);
   __shared__ u32 hist[4][256];
-  __shared__ u32 bucket[256];
   __shared__ int red[32];
   __shared__ i64 wsum[32];
   __shared__ int seg_end;
@@ -151,7 +158,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
       }
       __syncthreads();
       const int seg_hi = seg_end;
-      const bool have_key = sort_segment(p, lo, seg_lo, seg_hi, passes, n <= 65536 && key_max < 65536, warp_cnt, bucket, hist);
+      const bool have_key = sort_segment(p, lo, seg_lo, seg_hi, passes, n <= 65536 && key_max < 65536, warp_cnt, warp_off, hist);
       __syncthreads();
       for (int j = seg_lo + tid; j < seg_hi; j += T) {
         const int idx = p.perm[lo + j];
@@ -204,6 +211,9 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
 
 cudaError_t kvs_launch_sort(const SortParams& p, int grid, cudaStream_t stream) {
   if (p.n_instances <= 0) return cudaSuccess;
-  k_stats_sort<<<grid, KVS_SORT_THREADS, 0, stream>>>(p);
+  constexpr size_t smem = 2 * WARPS * 256 * sizeof(u32);   // digit counts and offsets per warp
+  const cudaError_t err = cudaFuncSetAttribute(k_stats_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (err != cudaSuccess) return err;
+  k_stats_sort<<<grid, KVS_SORT_THREADS, smem, stream>>>(p);
   return cudaGetLastError();
 }
