@@ -8,8 +8,9 @@
 //
 // Each pass ranks one tile of 1024 jobs at a time: lanes with equal digits find each other with
 // a warp match, per-warp digit counts go to shared memory, one column scan per digit turns them
-// into offsets behind the running bucket position.  Keys are re-read through the permutation
-// (they stay in L2 for instances of this size), so only 4 bytes per job move per pass.
+// into offsets behind the running bucket position.  Only 4 bytes per job move per pass: the
+// index, together with the key in the upper half of the word when both fit 16 bits; otherwise the
+// next pass re-reads the key through the index.
 #include "kvs_internal.cuh"
 
 namespace {
