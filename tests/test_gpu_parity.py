@@ -113,6 +113,24 @@ def test_large_single_instance(par):
     par.check_batch(inst, st, want_runs=False, label="big")
 
 
+def test_many_runs_per_round_over_several_tiles(par):
+    """Short prompts and a budget of some ten thousand tokens: the early phases of the geometric
+    families start eight or more runs per round (k >= 8 tau) and, with 150,000 jobs, still last
+    several tiles of rounds; with estimates both families carry killed jobs over."""
+    g = torch.Generator().manual_seed(77)
+    n = 150_000
+    s = torch.randint(0, 4, (n,), generator=g, dtype=torch.int32)
+    short = torch.randint(1, 41, (n,), generator=g, dtype=torch.int32)
+    long_ = torch.randint(41, 401, (n,), generator=g, dtype=torch.int32)
+    o = torch.where(torch.rand(n, generator=g) < 0.6, short, long_)
+    inst = workloads.Instances(torch.tensor([0, n], dtype=torch.int64), s, o)
+    st = binding.settings_grid([0], ["GBA", "GSA"], [35_003, 9_001, 300_007])
+    par.check_batch(inst, st, want_runs=False, label="many runs per round")
+    noise = torch.exp(0.5 * torch.randn(n, generator=g, dtype=torch.float64))
+    inst.o_est = torch.clamp(torch.round(o.to(torch.float64) * noise), 1, 400).to(torch.int32)
+    par.check_batch(inst, binding.settings_grid([0], ["GBA", "GSA"], [35_003]), want_runs=False, label="many runs per round, estimates")
+
+
 def test_empty_and_degenerate(par):
     off = torch.tensor([0, 0, 1, 1, 4], dtype=torch.int64)
     inst = workloads.Instances(off, torch.tensor([5, 0, 0, 0], dtype=torch.int32), torch.tensor([3, 1, 1, 1], dtype=torch.int32))
