@@ -72,7 +72,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
   L.lists = take(static_cast<size_t>(grid) * static_cast<size_t>(KVS_CTA_SCRATCH(max_n)));
   L.fin_rank = take(static_cast<size_t>(grid) * static_cast<size_t>(max_n) * 4);
-  L.counter = take(64);   // work counters of the three kernels, lengths of the two hand-over lists
+  L.counter = take(128);  // work counters of the kernels, lengths of the evaluation lists
   L.slow_list = take(static_cast<size_t>(P) * 8);
   L.walk_list = take(static_cast<size_t>(P) * 8);
   L.light_list = take(static_cast<size_t>(P) * 8);
@@ -268,11 +268,23 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     // Longest first: the rounds of a schedule grow as the budget shrinks and the slicing algorithm
     // visits more runs than the batching one, and the CTAs draw evaluations in list order, so this
     // order keeps the last CTAs from finishing a long evaluation alone.
+    // Without estimates the two geometric families have their own instantiation of the full variant
+    // and their own part of the list: the slicing algorithm first, then the batching one.
+    const bool split = inst->o_est == nullptr;
     std::stable_sort(ids.begin(), ids.begin() + n_full, [&](int64_t a, int64_t b) {
+      if (split && settings[a].family != settings[b].family) return settings[a].family > settings[b].family;
       if (settings[a].M != settings[b].M) return settings[a].M < settings[b].M;
       return settings[a].family > settings[b].family;
     });
-    const unsigned long long init[8] = {0, 0, 0, static_cast<unsigned long long>(n_full), 0, static_cast<unsigned long long>(n_light), 0, 0};
+    int64_t n_gsa = 0;
+    if (split) while (n_gsa < n_full && settings[ids[static_cast<size_t>(n_gsa)]].family == KVS_GSA) ++n_gsa;
+    const int64_t n_gba = split ? n_full - n_gsa : 0;
+    // [0] light work, [1] left-over count, [2] general work, [3] length of the full variant's list,
+    // [4] full work (starts behind the evaluations the two family kernels take), [5] light count,
+    // [6] [7] work and count of the slicing kernel, [8] [9] of the batching kernel
+    const unsigned long long init[16] = {0, 0, 0, static_cast<unsigned long long>(n_full), static_cast<unsigned long long>(n_gsa + n_gba),
+                                         static_cast<unsigned long long>(n_light), 0, static_cast<unsigned long long>(n_gsa),
+                                         0, static_cast<unsigned long long>(n_gba), 0, 0, 0, 0, 0, 0};
     if ((ce = cudaMemcpyAsync(counters, init, sizeof(init), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
         (n_full && (ce = cudaMemcpyAsync(ws + L.walk_list, ids.data(), static_cast<size_t>(n_full) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) ||
         (n_light && (ce = cudaMemcpyAsync(ws + L.light_list, ids.data() + n_full, static_cast<size_t>(n_light) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess))
@@ -285,15 +297,32 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
       bp.counter = counters;
       bp.eval_list = reinterpret_cast<const i64*>(ws + L.light_list);
       bp.eval_count = counters + 5;
-      ce = kvs_launch_fused(bp, grid_for(ctx->light_ctas_per_sm), 1, ctx->stream);
+      ce = kvs_launch_fused(bp, grid_for(ctx->light_ctas_per_sm), 1, KVS_FUSED_ANY, ctx->stream);
       if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
     }
     if (ctx->timing && !rg) cudaEventRecord(ctx->ev[3], ctx->stream);
-    bp.counter = counters + 4;
-    bp.eval_list = bp.walk_list;
-    bp.eval_count = bp.walk_count;
-    ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, ctx->stream);
-    if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    if (n_gsa) {
+      bp.counter = counters + 6;
+      bp.eval_list = bp.walk_list;
+      bp.eval_count = counters + 7;
+      ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, KVS_FUSED_GSA, ctx->stream);
+      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    }
+    if (n_gba) {
+      bp.counter = counters + 8;
+      bp.eval_list = bp.walk_list + n_gsa;
+      bp.eval_count = counters + 9;
+      ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, KVS_FUSED_GBA, ctx->stream);
+      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    }
+    if (n_light || n_full > n_gsa + n_gba) {
+      // what the light variant passed on, and the geometric evaluations of a call with estimates
+      bp.counter = counters + 4;
+      bp.eval_list = bp.walk_list;
+      bp.eval_count = bp.walk_count;
+      ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, KVS_FUSED_ANY, ctx->stream);
+      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    }
     bp.eval_list = bp.slow_list;
     bp.eval_count = bp.slow_count;
   }

@@ -791,7 +791,10 @@ struct FAcc {
 // LIGHT: the variant for evaluations that walk no rounds (schedule only, or SPS / SimS whose peak
 // comes from the run ends): no ring in shared memory and fewer registers, so that three CTAs fit an
 // SM; an evaluation that needs its rounds walked is passed on to the full variant through a list.
-template <bool LIGHT>
+// FAM: KVS_FUSED_ANY takes any evaluation; KVS_FUSED_GBA / KVS_FUSED_GSA are compiled for the batching /
+// slicing algorithm on exact response lengths only (the caller lists nothing else for them), so that
+// each keeps just its own paths and gets its own register allocation.
+template <bool LIGHT, int FAM>
 __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 1 : KVS_EVAL_MIN_CTAS) k_fused_eval(BuildParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   FShared& sh = *reinterpret_cast<FShared*>(smem_raw);
@@ -825,10 +828,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
     const i64 M = st.M;
     const i64 s_bar = st.s_bar >= 0 ? st.s_bar : stats.s_max;
     const i64 X = M - s_bar;
-    const int family = st.family;
+    const int family = FAM == KVS_FUSED_ANY ? st.family : (FAM == KVS_FUSED_GBA ? KVS_GBA : KVS_GSA);
     const bool geometric = family == KVS_GBA || family == KVS_GSA;
     const bool sim = family == KVS_SIMS;
-    const bool est = p.key != nullptr;
+    const bool est = FAM == KVS_FUSED_ANY && p.key != nullptr;
     const bool keyed = !(family == KVS_GSA && !est);          // plain GSA keeps the index order
     const bool carry = geometric && (family == KVS_GSA || est);
     const bool est_class = est && family == KVS_GBA;          // classes by the clipped estimate
@@ -1387,28 +1390,36 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
 
 static size_t fused_smem_bytes(bool light) { return light ? offsetof(FShared, dA) : sizeof(FShared); }
 
-template <bool LIGHT>
+template <bool LIGHT, int FAM>
 static int ctas_per_sm() {
   int n = 0;
-  cudaFuncSetAttribute(k_fused_eval<LIGHT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(LIGHT)));
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_fused_eval<LIGHT>, KVS_EVAL_THREADS, fused_smem_bytes(LIGHT)) != cudaSuccess) n = 1;
+  cudaFuncSetAttribute(k_fused_eval<LIGHT, FAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(LIGHT)));
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_fused_eval<LIGHT, FAM>, KVS_EVAL_THREADS, fused_smem_bytes(LIGHT)) != cudaSuccess) n = 1;
   return n < 1 ? 1 : n;
 }
 
-int kvs_fused_ctas_per_sm(int light) { return light ? ctas_per_sm<true>() : ctas_per_sm<false>(); }
+// CTAs per SM that every instantiation used for this kind of launch reaches.
+int kvs_fused_ctas_per_sm(int light) {
+  if (light) return ctas_per_sm<true, KVS_FUSED_ANY>();
+  const int a = ctas_per_sm<false, KVS_FUSED_ANY>(), b = ctas_per_sm<false, KVS_FUSED_GBA>(), c = ctas_per_sm<false, KVS_FUSED_GSA>();
+  return a < b ? (a < c ? a : c) : (b < c ? b : c);
+}
 
-// The caller zeroes the counters.  light: the variant without the ring (see k_fused_eval).
-cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, cudaStream_t stream) {
-  if (p.P <= 0) return cudaSuccess;
-  cudaError_t err;
-  if (light) {
-    err = cudaFuncSetAttribute(k_fused_eval<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(true)));
-    if (err != cudaSuccess) return err;
-    k_fused_eval<true><<<grid, KVS_EVAL_THREADS, fused_smem_bytes(true), stream>>>(p);
-  } else {
-    err = cudaFuncSetAttribute(k_fused_eval<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(false)));
-    if (err != cudaSuccess) return err;
-    k_fused_eval<false><<<grid, KVS_EVAL_THREADS, fused_smem_bytes(false), stream>>>(p);
-  }
+template <bool LIGHT, int FAM>
+static cudaError_t launch(const BuildParams& p, int grid, cudaStream_t stream) {
+  const cudaError_t err = cudaFuncSetAttribute(k_fused_eval<LIGHT, FAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem_bytes(LIGHT)));
+  if (err != cudaSuccess) return err;
+  k_fused_eval<LIGHT, FAM><<<grid, KVS_EVAL_THREADS, fused_smem_bytes(LIGHT), stream>>>(p);
   return cudaGetLastError();
+}
+
+// The caller zeroes the counters.  light: the variant without the ring (see k_fused_eval); fam: one of
+// KVS_FUSED_ANY / KVS_FUSED_GBA / KVS_FUSED_GSA (the last two for the full variant only, and only for
+// lists of that family in a call without estimates).
+cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam, cudaStream_t stream) {
+  if (p.P <= 0) return cudaSuccess;
+  if (light) return launch<true, KVS_FUSED_ANY>(p, grid, stream);
+  if (fam == KVS_FUSED_GBA) return launch<false, KVS_FUSED_GBA>(p, grid, stream);
+  if (fam == KVS_FUSED_GSA) return launch<false, KVS_FUSED_GSA>(p, grid, stream);
+  return launch<false, KVS_FUSED_ANY>(p, grid, stream);
 }
