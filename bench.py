@@ -301,13 +301,16 @@ def run_ours(args):
     traffic = None
     if name == "c5" and geo and C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION:
         traffic = C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION * geo
-    # kernels of one kvs_evaluate_built call: ordering kernel, light variant (SPS / SimS), one full-variant
-    # launch per geometric family (a single one for all of them when estimates are given), the full variant
-    # for what the light one passes on, and the general kernel on the left-over list
-    has_light = any(f in ("SPS", "SIMS") for f in fams)
+    # kernels of one kvs_evaluate_built call: ordering kernel; without estimates one launch of the light
+    # variant per SPS / SimS family and one of the full variant per geometric family (with estimates one of
+    # each for all families); the full variant for what the light one passes on; the general kernel on the
+    # left-over list
+    n_light_fams = sum(f in ("SPS", "SIMS") for f in fams)
     n_geo_fams = sum(f in ("GBA", "GSA") for f in fams)
-    with_est = inst.o_est is not None
-    launches_per_step = 1 + int(has_light) + (n_geo_fams if not with_est else 0) + int(has_light or (with_est and n_geo_fams > 0)) + 1
+    if inst.o_est is None:
+        launches_per_step = 1 + n_light_fams + n_geo_fams + int(n_light_fams > 0) + 1
+    else:
+        launches_per_step = 1 + int(n_light_fams > 0) + int(n_light_fams + n_geo_fams > 0) + 1
     line = {
         "metric": METRIC, "value": steps_all / sec_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * sec_per_step, "higher_is_better": True, "scaling": "weak",

@@ -72,7 +72,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   const int64_t grid = P < KVS_MAX_GRID ? P : KVS_MAX_GRID;
   L.lists = take(static_cast<size_t>(grid) * static_cast<size_t>(KVS_CTA_SCRATCH(max_n)));
   L.fin_rank = take(static_cast<size_t>(grid) * static_cast<size_t>(max_n) * 4);
-  L.counter = take(128);  // work counters of the kernels, lengths of the evaluation lists
+  L.counter = take(256);  // work counters of the kernels, lengths of the evaluation lists
   L.slow_list = take(static_cast<size_t>(P) * 8);
   L.walk_list = take(static_cast<size_t>(P) * 8);
   L.light_list = take(static_cast<size_t>(P) * 8);
@@ -268,23 +268,33 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     // Longest first: the rounds of a schedule grow as the budget shrinks and the slicing algorithm
     // visits more runs than the batching one, and the CTAs draw evaluations in list order, so this
     // order keeps the last CTAs from finishing a long evaluation alone.
-    // Without estimates the two geometric families have their own instantiation of the full variant
-    // and their own part of the list: the slicing algorithm first, then the batching one.
+    // Without estimates every family has its own instantiation of the kernel and its own part of the
+    // list: in the full variant the slicing algorithm first, then the batching one.
     const bool split = inst->o_est == nullptr;
     std::stable_sort(ids.begin(), ids.begin() + n_full, [&](int64_t a, int64_t b) {
       if (split && settings[a].family != settings[b].family) return settings[a].family > settings[b].family;
       if (settings[a].M != settings[b].M) return settings[a].M < settings[b].M;
       return settings[a].family > settings[b].family;
     });
-    int64_t n_gsa = 0;
-    if (split) while (n_gsa < n_full && settings[ids[static_cast<size_t>(n_gsa)]].family == KVS_GSA) ++n_gsa;
-    const int64_t n_gba = split ? n_full - n_gsa : 0;
-    // [0] light work, [1] left-over count, [2] general work, [3] length of the full variant's list,
-    // [4] full work (starts behind the evaluations the two family kernels take), [5] light count,
-    // [6] [7] work and count of the slicing kernel, [8] [9] of the batching kernel
-    const unsigned long long init[16] = {0, 0, 0, static_cast<unsigned long long>(n_full), static_cast<unsigned long long>(n_gsa + n_gba),
-                                         static_cast<unsigned long long>(n_light), 0, static_cast<unsigned long long>(n_gsa),
-                                         0, static_cast<unsigned long long>(n_gba), 0, 0, 0, 0, 0, 0};
+    if (split)
+      std::stable_sort(ids.begin() + n_full, ids.end(), [&](int64_t a, int64_t b) { return settings[a].family < settings[b].family; });
+    int64_t full_of[4] = {0, 0, 0, 0}, light_of[4] = {0, 0, 0, 0};
+    if (split) {
+      for (int64_t i = 0; i < n_full; ++i) ++full_of[settings[ids[static_cast<size_t>(i)]].family];
+      for (int64_t i = n_full; i < P; ++i) ++light_of[settings[ids[static_cast<size_t>(i)]].family];
+    }
+    // [1] left-over count, [2] general work, [3] length of the full variant's list, [4] work of the full
+    // variant for any family (starts behind the evaluations the family kernels take), [6] [7] work and
+    // count of the light variant for any family, [8 + 2f] [9 + 2f] of the light kernel of family f,
+    // [16 + 2f] [17 + 2f] of the full kernel of family f
+    unsigned long long init[32] = {};
+    init[3] = static_cast<unsigned long long>(n_full);
+    init[4] = static_cast<unsigned long long>(split ? n_full : 0);
+    init[7] = static_cast<unsigned long long>(split ? 0 : n_light);
+    for (int f = 0; f < 4; ++f) {
+      init[9 + 2 * f] = static_cast<unsigned long long>(light_of[f]);
+      init[17 + 2 * f] = static_cast<unsigned long long>(full_of[f]);
+    }
     if ((ce = cudaMemcpyAsync(counters, init, sizeof(init), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
         (n_full && (ce = cudaMemcpyAsync(ws + L.walk_list, ids.data(), static_cast<size_t>(n_full) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess) ||
         (n_light && (ce = cudaMemcpyAsync(ws + L.light_list, ids.data() + n_full, static_cast<size_t>(n_light) * 8, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess))
@@ -293,29 +303,41 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     bp.slow_list = reinterpret_cast<i64*>(ws + L.slow_list);
     bp.walk_count = counters + 3;
     bp.walk_list = reinterpret_cast<i64*>(ws + L.walk_list);
-    if (n_light) {
-      bp.counter = counters;
-      bp.eval_list = reinterpret_cast<const i64*>(ws + L.light_list);
-      bp.eval_count = counters + 5;
+    const i64* const light_list = reinterpret_cast<const i64*>(ws + L.light_list);
+    if (split) {
+      int64_t at = 0;
+      for (int f = 0; f < 4; ++f) {
+        if (light_of[f]) {
+          bp.counter = counters + 8 + 2 * f;
+          bp.eval_list = light_list + at;
+          bp.eval_count = counters + 9 + 2 * f;
+          ce = kvs_launch_fused(bp, grid_for(ctx->light_ctas_per_sm), 1, f, ctx->stream);
+          if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+        }
+        at += light_of[f];
+      }
+    } else if (n_light) {
+      bp.counter = counters + 6;
+      bp.eval_list = light_list;
+      bp.eval_count = counters + 7;
       ce = kvs_launch_fused(bp, grid_for(ctx->light_ctas_per_sm), 1, KVS_FUSED_ANY, ctx->stream);
       if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
     }
     if (ctx->timing && !rg) cudaEventRecord(ctx->ev[3], ctx->stream);
-    if (n_gsa) {
-      bp.counter = counters + 6;
-      bp.eval_list = bp.walk_list;
-      bp.eval_count = counters + 7;
-      ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, KVS_FUSED_GSA, ctx->stream);
-      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+    if (split) {
+      int64_t at = 0;
+      for (int f = KVS_GSA; f >= KVS_GBA; --f) {   // the order of the list
+        if (full_of[f]) {
+          bp.counter = counters + 16 + 2 * f;
+          bp.eval_list = bp.walk_list + at;
+          bp.eval_count = counters + 17 + 2 * f;
+          ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, f, ctx->stream);
+          if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
+        }
+        at += full_of[f];
+      }
     }
-    if (n_gba) {
-      bp.counter = counters + 8;
-      bp.eval_list = bp.walk_list + n_gsa;
-      bp.eval_count = counters + 9;
-      ce = kvs_launch_fused(bp, grid_for(ctx->fused_ctas_per_sm), 0, KVS_FUSED_GBA, ctx->stream);
-      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "fused launch");
-    }
-    if (n_light || n_full > n_gsa + n_gba) {
+    if (n_light || (!split && n_full)) {
       // what the light variant passed on, and the geometric evaluations of a call with estimates
       bp.counter = counters + 4;
       bp.eval_list = bp.walk_list;

@@ -791,8 +791,8 @@ struct FAcc {
 // LIGHT: the variant for evaluations that walk no rounds (schedule only, or SPS / SimS whose peak
 // comes from the run ends): no ring in shared memory and fewer registers, so that three CTAs fit an
 // SM; an evaluation that needs its rounds walked is passed on to the full variant through a list.
-// FAM: KVS_FUSED_ANY takes any evaluation; KVS_FUSED_GBA / KVS_FUSED_GSA are compiled for the batching /
-// slicing algorithm on exact response lengths only (the caller lists nothing else for them), so that
+// FAM: KVS_FUSED_ANY takes any evaluation; a family id (KVS_GBA .. KVS_SIMS) gives the kernel compiled
+// for that family on exact response lengths only (the caller lists nothing else for it), so that
 // each keeps just its own paths and gets its own register allocation.
 template <bool LIGHT, int FAM>
 __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 1 : KVS_EVAL_MIN_CTAS) k_fused_eval(BuildParams p) {
@@ -828,7 +828,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
     const i64 M = st.M;
     const i64 s_bar = st.s_bar >= 0 ? st.s_bar : stats.s_max;
     const i64 X = M - s_bar;
-    const int family = FAM == KVS_FUSED_ANY ? st.family : (FAM == KVS_FUSED_GBA ? KVS_GBA : KVS_GSA);
+    const int family = FAM == KVS_FUSED_ANY ? st.family : FAM;
     const bool geometric = family == KVS_GBA || family == KVS_GSA;
     const bool sim = family == KVS_SIMS;
     const bool est = FAM == KVS_FUSED_ANY && p.key != nullptr;
@@ -1400,9 +1400,14 @@ static int ctas_per_sm() {
 
 // CTAs per SM that every instantiation used for this kind of launch reaches.
 int kvs_fused_ctas_per_sm(int light) {
-  if (light) return ctas_per_sm<true, KVS_FUSED_ANY>();
-  const int a = ctas_per_sm<false, KVS_FUSED_ANY>(), b = ctas_per_sm<false, KVS_FUSED_GBA>(), c = ctas_per_sm<false, KVS_FUSED_GSA>();
-  return a < b ? (a < c ? a : c) : (b < c ? b : c);
+  int n;
+  if (light) {
+    n = ctas_per_sm<true, KVS_FUSED_ANY>();
+    n = min(n, min(min(ctas_per_sm<true, KVS_GBA>(), ctas_per_sm<true, KVS_GSA>()), min(ctas_per_sm<true, KVS_SPS>(), ctas_per_sm<true, KVS_SIMS>())));
+  } else {
+    n = min(ctas_per_sm<false, KVS_FUSED_ANY>(), min(ctas_per_sm<false, KVS_GBA>(), ctas_per_sm<false, KVS_GSA>()));
+  }
+  return n;
 }
 
 template <bool LIGHT, int FAM>
@@ -1413,13 +1418,21 @@ static cudaError_t launch(const BuildParams& p, int grid, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-// The caller zeroes the counters.  light: the variant without the ring (see k_fused_eval); fam: one of
-// KVS_FUSED_ANY / KVS_FUSED_GBA / KVS_FUSED_GSA (the last two for the full variant only, and only for
-// lists of that family in a call without estimates).
+// The caller zeroes the counters.  light: the variant without the ring (see k_fused_eval); fam:
+// KVS_FUSED_ANY, or a family id for a list of that family alone in a call without estimates (the
+// full variant has such kernels for the two geometric families, the light one for all four).
 cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam, cudaStream_t stream) {
   if (p.P <= 0) return cudaSuccess;
-  if (light) return launch<true, KVS_FUSED_ANY>(p, grid, stream);
-  if (fam == KVS_FUSED_GBA) return launch<false, KVS_FUSED_GBA>(p, grid, stream);
-  if (fam == KVS_FUSED_GSA) return launch<false, KVS_FUSED_GSA>(p, grid, stream);
+  if (light) {
+    switch (fam) {
+      case KVS_GBA: return launch<true, KVS_GBA>(p, grid, stream);
+      case KVS_GSA: return launch<true, KVS_GSA>(p, grid, stream);
+      case KVS_SPS: return launch<true, KVS_SPS>(p, grid, stream);
+      case KVS_SIMS: return launch<true, KVS_SIMS>(p, grid, stream);
+      default: return launch<true, KVS_FUSED_ANY>(p, grid, stream);
+    }
+  }
+  if (fam == KVS_GBA) return launch<false, KVS_GBA>(p, grid, stream);
+  if (fam == KVS_GSA) return launch<false, KVS_GSA>(p, grid, stream);
   return launch<false, KVS_FUSED_ANY>(p, grid, stream);
 }

@@ -122,7 +122,7 @@ struct SweepParams {
 cudaError_t kvs_launch_sort(const SortParams& p, int grid, cudaStream_t stream);
 cudaError_t kvs_launch_build(const BuildParams& p, int grid, cudaStream_t stream);
 int kvs_build_ctas_per_sm();
-enum { KVS_FUSED_ANY = -1, KVS_FUSED_GBA = 0, KVS_FUSED_GSA = 1 };   // instantiations of the fast kernel
+enum { KVS_FUSED_ANY = -1 };   // instantiation of the fast kernel for any family; the others are named by the family id
 cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam, cudaStream_t stream);
 int kvs_fused_ctas_per_sm(int light);
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
