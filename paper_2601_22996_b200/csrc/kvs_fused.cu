@@ -1060,60 +1060,107 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
         }
       } else {
         // The rank of a job in the phase that completes it = positions before it that leave in that
-        // phase or later: the table gives the count before the segment, ballots the rest.
+        // phase or later: the table gives the count before the segment; inside the segment a lane
+        // holds the classes of eight consecutive positions, and for every class q present one byte
+        // compare per lane and one warp scan count the positions with class >= q before each lane.
+        const bool vec_o = (reinterpret_cast<uintptr_t>(O_ord + seg_lo) & 15u) == 0;
         for (int seg = warp; seg < nsegs; seg += WARPS) {
-        u32 g0 = lane < L ? G[seg * L + lane] : 0u;
-        u32 g1 = lane + 32 < L ? G[seg * L + lane + 32] : 0u;
-        u32 g2 = lane + 64 < L ? G[seg * L + lane + 64] : 0u;
-        const int x1 = min(nseg, (seg + 1) * SEG);
-        for (int xb = seg * SEG; xb < x1; xb += 32) {
-          const int x = xb + lane;
-          const bool valid = x < x1;
-          u32 ov = 0;
-          int l = 0, f = 0;
-          if (valid) {
-            ov = static_cast<u32>(__ldg(O_ord + seg_lo + x));
-            if (est_class) {
-              const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + x)), Xc);
-              f = pow2 ? class_pow2(Xc, kc) : class_of(sh.tau, L, kc);
-            }
-            l = cls[x];
+          const int xb = seg * SEG + 8 * lane;
+          const int room = nseg - xb;
+          const u32 lim = room >= 8 ? 0xffu : (room > 0 ? (1u << room) - 1u : 0u);
+          u32 ov_[8];
+          if (vec_o && room >= 8) {
+            const uint4 b0 = __ldg(reinterpret_cast<const uint4*>(O_ord + seg_lo + xb));
+            const uint4 b1 = __ldg(reinterpret_cast<const uint4*>(O_ord + seg_lo + xb) + 1);
+            ov_[0] = b0.x; ov_[1] = b0.y; ov_[2] = b0.z; ov_[3] = b0.w; ov_[4] = b1.x; ov_[5] = b1.y; ov_[6] = b1.z; ov_[7] = b1.w;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ov_[j] = (lim >> j & 1u) ? static_cast<u32>(__ldg(O_ord + seg_lo + xb + j)) : 0u;
           }
-          const u32 vm = __ballot_sync(0xffffffffu, valid);
-          const int nvalid = __popc(vm);
-          const int pmin = __reduce_min_sync(0xffffffffu, valid ? l : 0x7fffffff);
-          const int pmax = __reduce_max_sync(0xffffffffu, valid ? l : 0);
-          u32 rank = 0;
+          const uint2 cw = *reinterpret_cast<const uint2*>(cls + xb);
+          // smallest and largest class among the warp's valid positions
+          u32 lo4 = 0xffu, hi4 = 0u;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const u32 c = ((j < 4 ? cw.x : cw.y) >> (8 * (j & 3))) & 0xffu;
+            if (lim >> j & 1u) { lo4 = min(lo4, c); hi4 = max(hi4, c); }
+          }
+          const int pmin = static_cast<int>(__reduce_min_sync(0xffffffffu, lo4));
+          const int pmax = static_cast<int>(__reduce_max_sync(0xffffffffu, hi4));
+          u32 rk_[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) rk_[j] = 0;
           for (int q = pmin; q <= pmax; ++q) {
-            const u32 m = __ballot_sync(0xffffffffu, valid && l >= q);
-            const u32 gs = q < 32 ? g0 : (q < 64 ? g1 : g2);
-            const u32 g = __shfl_sync(0xffffffffu, gs, q & 31);
-            if (l == q) rank = g + __popc(m & lanemask_lt());
-            if (lane == (q & 31)) {
-              const u32 c = __popc(m);
-              if (q < 32) g0 += c; else if (q < 64) g1 += c; else g2 += c;
+            const u32 p4 = static_cast<u32>(q) * 0x01010101u;
+            const u32 ge = (byte_mask4(cw.x, p4, true) | byte_mask4(cw.y, p4, true) << 4) & lim;
+            const u32 eq = (byte_mask4(cw.x, p4, false) | byte_mask4(cw.y, p4, false) << 4) & lim;
+            const u32 cnt = static_cast<u32>(__popc(ge));
+            u32 incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+              const u32 y = __shfl_up_sync(0xffffffffu, incl, d);
+              if (lane >= d) incl += y;
+            }
+            if (eq) {
+              const u32 before = G[seg * L + q] + incl - cnt;
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                if (eq >> j & 1u) rk_[j] = before + static_cast<u32>(__popc(ge & ((1u << j) - 1u)));
             }
           }
-          // every valid position counts for the phases before the smallest class seen
-          if (lane < pmin) g0 += nvalid;
-          if (lane + 32 < pmin) g1 += nvalid;
-          if (lane + 64 < pmin) g2 += nvalid;
-          if (valid) {
-            const u32 tau = sh.tau[l], k = sh.k[l];
-            const u32 stt = sh.pbase[l] + slot_mul(rank, tau, k, sh.kinv[l]);
-            acc.steps += ov + (sh.taupre[l] - sh.taupre[f]);
-            if (keyed) {
-              fin_start[seg_lo + x] = stt;
+          u32 st_[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            st_[j] = 0;
+            if (lim >> j & 1u) {
+              const int l = static_cast<int>(((j < 4 ? cw.x : cw.y) >> (8 * (j & 3))) & 0xffu);
+              int f = 0;
+              if (est_class) {
+                const u32 kc = min(static_cast<u32>(__ldg(K_ord + seg_lo + xb + j)), Xc);
+                f = pow2 ? class_pow2(Xc, kc) : class_of(sh.tau, L, kc);
+              }
+              const u32 tau = sh.tau[l], k = sh.k[l];
+              st_[j] = sh.pbase[l] + slot_mul(rk_[j], tau, k, sh.kinv[l]);
+              acc.steps += ov_[j] + (sh.taupre[l] - sh.taupre[f]);
+            }
+          }
+          if (keyed) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (lim >> j & 1u) fin_start[seg_lo + xb + j] = st_[j];
+          } else {
+            const bool vec_out = room >= 8 && ((seg_lo + xb) & 3) == 0 &&
+                                 ((reinterpret_cast<uintptr_t>(out_start) | reinterpret_cast<uintptr_t>(out_done)) & 15u) == 0;
+            u32 dn_[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              dn_[j] = st_[j] + ov_[j];
+              if (lim >> j & 1u) {
+                acc.hmax = max(acc.hmax, dn_[j]);
+                acc.flow += static_cast<u64>(static_cast<i64>(dn_[j]) - (ARR ? __ldg(ARR + seg_lo + xb + j) : 0));
+              }
+            }
+            if (vec_out) {
+              if (out_start) {
+                int4* const d = reinterpret_cast<int4*>(out_start + seg_lo + xb);
+                __stcs(d, make_int4(static_cast<int>(st_[0]), static_cast<int>(st_[1]), static_cast<int>(st_[2]), static_cast<int>(st_[3])));
+                __stcs(d + 1, make_int4(static_cast<int>(st_[4]), static_cast<int>(st_[5]), static_cast<int>(st_[6]), static_cast<int>(st_[7])));
+              }
+              if (out_done) {
+                int4* const d = reinterpret_cast<int4*>(out_done + seg_lo + xb);
+                __stcs(d, make_int4(static_cast<int>(dn_[0]), static_cast<int>(dn_[1]), static_cast<int>(dn_[2]), static_cast<int>(dn_[3])));
+                __stcs(d + 1, make_int4(static_cast<int>(dn_[4]), static_cast<int>(dn_[5]), static_cast<int>(dn_[6]), static_cast<int>(dn_[7])));
+              }
             } else {
-              const int j = seg_lo + x;
-              const u32 done = stt + ov;
-              acc.hmax = max(acc.hmax, done);
-              acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
-              if (out_start) __stcs(&out_start[j], static_cast<int32_t>(stt));
-              if (out_done) __stcs(&out_done[j], static_cast<int32_t>(done));
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                if (lim >> j & 1u) {
+                  if (out_start) __stcs(&out_start[seg_lo + xb + j], static_cast<int32_t>(st_[j]));
+                  if (out_done) __stcs(&out_done[seg_lo + xb + j], static_cast<int32_t>(dn_[j]));
+                }
+              }
             }
           }
-        }
         }
         if (keyed) {
           __syncthreads();
