@@ -27,10 +27,10 @@ from paper_2601_22996_b200 import workloads  # noqa: E402
 METRIC, UNIT = "schedule_evaluation_job_steps_per_sec", "job-steps/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, the full variant of
 # k_fused_eval (it takes the geometric evaluations), from the ncu capture summarised in
-# profiles/k_fused_eval_c5.md (592 instances of config 5: 1,184 GBA/GSA evaluations, 3.228 GB).
+# profiles/k_fused_eval_c5.md (592 instances of config 5: 1,184 GBA/GSA evaluations, 3.418 GB, the launches of the two families together).
 # Traffic grows with the number of evaluations (each CTA works on one at a time), so a launch is scaled
 # by its evaluation count.  Valid for the kernel state named in that file; set to None when the kernel changes.
-C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION = 3.228184e9 / 1184
+C5_TRAFFIC_BYTES_PER_GEOMETRIC_EVALUATION = 3.418012e9 / 1184
 WORKLOADS = {
     # name: (generator, instances, jobs per instance, families, description)
     "c2": ("config2", 1024, 10_000, ["GBA", "GSA"], "config 2: 1,024 instances x 10,000 jobs, M in {2^17..2^24}, GBA+GSA"),
