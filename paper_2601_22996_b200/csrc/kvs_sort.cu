@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(KVS_SORT_THREADS) k_stats_sort(SortParams p) {
         __syncthreads();
         if (lane_id() == 31) wsum[tid >> 5] = incl;
         __syncthreads();
-        const i64 w = wsum[lane_id()];
+        const i64 w = static_cast<int>(lane_id()) < WARPS ? wsum[lane_id()] : 0;
         i64 wi = w;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
