@@ -211,9 +211,14 @@ int kvs_evaluate_schedule(kvs_ctx* ctx, const kvs_runs* runs, const kvs_eval_out
  * in `err` (optional buffer of err_len bytes).  The call itself allocates nothing (no cudaMalloc,
  * no cudaFree, no allocating library routine).
  * The first call on each device looks up the array's device address; make that first call
- * before any stream capture.  All calls on a device share the array: each call clears the part
- * it uses, so results do not depend on earlier calls, but calls that overlap on the GPU (two
- * streams, two threads) race - serialise them.  Outputs and status bits as kvs_evaluate_schedule. */
+ * before any stream capture (the look-up is safe against another host thread doing the same).
+ * The work is issued with `device` current; the caller's current device is restored on return.
+ * All calls on a device share the array: each call clears the part it uses, so results do not
+ * depend on earlier calls, but calls that overlap on the GPU (two streams, two threads) race -
+ * serialise them.  Outputs and status bits as kvs_evaluate_schedule.  The kernel trusts no host
+ * copy: an evaluation whose DEVICE offsets profile_off[e], profile_off[e + 1] are not monotone or
+ * reach beyond `capacity_total` is skipped with KVS_EVAL_CAPACITY | KVS_EVAL_BAD_INPUT in
+ * status[e] (peak -1, other scalars 0) and nothing of it is written. */
 int kvs_evaluate_schedule_noalloc(int32_t device, void* stream, const kvs_runs* runs,
                                   const kvs_eval_out* ev, int64_t capacity_total,
                                   char* err, uint64_t err_len);

@@ -620,6 +620,7 @@ int kvs_evaluate_schedule(kvs_ctx* ctx, const kvs_runs* runs, const kvs_eval_out
   gp.runs = *runs; gp.ev = *ev;
   gp.dconst = reinterpret_cast<i64*>(ws);
   gp.dcount = reinterpret_cast<int32_t*>(ws + need_a);
+  gp.slots = cap_total + runs->P;
   ce = cudaMemsetAsync(ws, 0, need, ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "memset");
   ce = kvs_launch_generic(gp, ctx->stream);

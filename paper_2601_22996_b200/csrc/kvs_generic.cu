@@ -6,6 +6,7 @@
 // in global memory (64-bit constant terms, 32-bit slopes), prefix-sums both tile by tile and
 // forms memory(t) = A(t) + t * B(t), its maximum, and the scalar reductions.  Nothing is assumed
 // about the order or overlap of the runs, so this path trades speed for generality.
+#include <atomic>
 #include <cstdio>
 
 #include "kvs_internal.cuh"
@@ -26,6 +27,20 @@ __global__ void __launch_bounds__(T) k_generic_eval(GenericParams p) {
     const i64 r0 = R.run_off[e], r1 = R.run_off[e + 1];
     const i64 pbase = p.ev.profile_off[e];
     const i64 cap = p.ev.profile_off[e + 1] - pbase;
+    // The difference arrays hold `slots` entries; evaluation e owns entries pbase + e .. pbase + e + cap.
+    // Offsets on the device that do not fit (not monotone, or larger than the host said when the arrays
+    // were sized) would send the atomics outside them: such an evaluation is reported and skipped.
+    if (pbase < 0 || cap < 0 || pbase > p.slots || cap > p.slots - pbase || e + 1 > p.slots - pbase - cap) {
+      if (tid == 0) {
+        if (p.ev.peak) p.ev.peak[e] = -1;
+        if (p.ev.flow) p.ev.flow[e] = 0;
+        if (p.ev.job_steps) p.ev.job_steps[e] = 0;
+        if (p.ev.horizon) p.ev.horizon[e] = 0;
+        if (p.ev.feasible) p.ev.feasible[e] = 0;
+        if (p.ev.status) p.ev.status[e] = KVS_EVAL_CAPACITY | KVS_EVAL_BAD_INPUT;
+      }
+      continue;
+    }
     i64* const dA = p.dconst + pbase + e;      // cap + 1 entries
     int32_t* const dB = p.dcount + pbase + e;
     i64 steps = 0, hmax = 0, flow = 0;
@@ -147,7 +162,9 @@ static __device__ __align__(256) unsigned char kvs_noalloc_scratch[KVS_NOALLOC_S
 
 namespace {
 constexpr int KVS_NOALLOC_MAX_DEVICES = 64;
-void* g_noalloc_ptr[KVS_NOALLOC_MAX_DEVICES] = {};   // device address of the array, per device
+// Device address of the array, per device.  Atomic, so that two host threads making their first call on
+// a device at the same time both end up with the same, fully written pointer.
+std::atomic<void*> g_noalloc_ptr[KVS_NOALLOC_MAX_DEVICES] = {};
 void put_msg(char* err, uint64_t len, const char* msg) {
   if (err && len) { snprintf(err, static_cast<size_t>(len), "%s", msg); }
 }
@@ -164,22 +181,29 @@ extern "C" int kvs_evaluate_schedule_noalloc(int32_t device, void* stream, const
     put_msg(err, err_len, "null run array or profile_off");
     return KVS_E_ARG;
   }
-  if (capacity_total + runs->P > KVS_NOALLOC_SLOTS) {
+  if (runs->P > KVS_NOALLOC_SLOTS || capacity_total > KVS_NOALLOC_SLOTS - runs->P) {
     put_msg(err, err_len, "capacity_total + P exceeds the 1,048,576 slots of the built-in scratch array; "
                           "use kvs_evaluate_schedule with a workspace instead");
     return KVS_E_CAPACITY;
   }
-  cudaError_t ce = cudaSetDevice(device);
+  // The work is issued with `device` current; the caller's current device is put back before returning.
+  int prev_device = -1;
+  cudaError_t ce = cudaGetDevice(&prev_device);
+  if (ce == cudaSuccess && prev_device != device) ce = cudaSetDevice(device);
   if (ce != cudaSuccess) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
-  if (!g_noalloc_ptr[device]) {
+  struct Restore {
+    int prev, cur;
+    ~Restore() { if (prev >= 0 && prev != cur) cudaSetDevice(prev); }
+  } restore{prev_device, device};
+  void* ptr = g_noalloc_ptr[device].load(std::memory_order_acquire);
+  if (!ptr) {
     // In host code the array's name is only a handle; its device address has to be asked for,
     // once per device, with that device current.
-    void* ptr = nullptr;
     ce = cudaGetSymbolAddress(&ptr, kvs_noalloc_scratch);
     if (ce != cudaSuccess || !ptr) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
-    g_noalloc_ptr[device] = ptr;
+    g_noalloc_ptr[device].store(ptr, std::memory_order_release);
   }
-  unsigned char* base = static_cast<unsigned char*>(g_noalloc_ptr[device]);
+  unsigned char* base = static_cast<unsigned char*>(ptr);
   const size_t slots = static_cast<size_t>(capacity_total + runs->P);
   const size_t bytes_a = (slots * 8 + 255) & ~static_cast<size_t>(255);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -190,6 +214,7 @@ extern "C" int kvs_evaluate_schedule_noalloc(int32_t device, void* stream, const
   gp.ev = *ev;
   gp.dconst = reinterpret_cast<i64*>(base);
   gp.dcount = reinterpret_cast<int32_t*>(base + bytes_a);
+  gp.slots = static_cast<i64>(slots);
   ce = kvs_launch_generic(gp, s);
   if (ce != cudaSuccess) { put_msg(err, err_len, cudaGetErrorString(ce)); return KVS_E_CUDA; }
   return KVS_OK;

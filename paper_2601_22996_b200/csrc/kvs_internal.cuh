@@ -103,6 +103,7 @@ struct GenericParams {
   kvs_eval_out ev;
   i64* dconst;              // [capacity_total + P] difference array of the constant terms
   int32_t* dcount;          // [capacity_total + P] difference array of the slopes
+  i64 slots;                // entries of each array; the kernel skips an evaluation whose offsets reach beyond
 };
 
 struct SweepParams {

@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    config.addinivalue_line("markers", "full: the pass over every evaluation of every config (KVS_FULL_VERIFY=1, -m full)")
 
 
 @pytest.fixture(scope="session")

@@ -278,6 +278,13 @@ def test_area_lower_bound_and_upper_bounds():
             assert gsa.flow <= gsa_bound
             assert gsa_bound <= (2 + 2 / (al - 1)) * upper_gba
             assert all(k[q] >= k[t] for q in range(len(k)) for t in range(q, len(k)))
+            # the oracle's bound evaluator returns exactly these integers (the sums above are written
+            # from the two packing-efficiency lemmas and the area lemma, not from its code)
+            x = [0] + tau[:-1]
+            area2 = [2 * s0 * x[p] + x[p] * (x[p] + 1) for p in range(len(tau))]
+            lower_2m = sum(area2[p] * (n_p[p] * (n_p[p] + 1) // 2 + n_gt[p] * n_p[p]) for p in range(len(tau)))
+            B = oracle.bounds(s, o, M, alpha=alpha)
+            assert (B.status, B.upper_gba, B.upper_gsa, B.lower_2m) == (0, upper_gba, gsa_bound, lower_2m)
 
 
 def test_ratios_against_bruteforce_optimum():
