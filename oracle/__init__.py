@@ -46,6 +46,8 @@ def lib():
         L.kvo_ladder.argtypes = [i64, i32, i32, i64, p, i64]
         L.kvo_build.restype = p
         L.kvo_build.argtypes = [i32, i64, p, p, p, p, i64, i32, i32, i64, i64, i64, i64, i64]
+        L.kvo_build_variant.restype = p
+        L.kvo_build_variant.argtypes = [i32, i64, p, p, p, p, i64, i32, i32, i64, i64, i64, i64, i64, i32, i32]
         L.kvo_free.argtypes = [p]
         L.kvo_scalars.argtypes = [p, p]
         L.kvo_jobs.argtypes = [p, p, p]
@@ -107,15 +109,18 @@ class Schedule:
 
 
 def build_schedule(family, s, o, M, *, o_est=None, arrival=None, alpha=(2, 1), beta0=0,
-                   s_bar=-1, tau=0, k=0, window=0) -> Schedule:
-    """Build one schedule for one instance (see ``kvo_build``)."""
+                   s_bar=-1, tau=0, k=0, window=0, subroutine=0, per_class_s=0) -> Schedule:
+    """Build one schedule for one instance (see ``kvo_build``).  ``subroutine=1`` runs the simultaneous
+    schedule inside every geometric phase, ``per_class_s=1`` sizes each phase's parallelism by the
+    longest prompt among its participants (see ``build`` in kvs_oracle.cpp)."""
     fam = FAMILY[family] if isinstance(family, str) else int(family)
     s_, o_ = _arr(s, np.int32), _arr(o, np.int32)
     e_, a_ = _arr(o_est, np.int32), _arr(arrival, np.int64)
     n = int(s_.shape[0])
     L = lib()
-    h = L.kvo_build(fam, n, _ptr(s_), _ptr(o_), _ptr(e_), _ptr(a_), int(M), int(alpha[0]),
-                    int(alpha[1]), int(beta0), int(s_bar), int(tau), int(k), int(window))
+    h = L.kvo_build_variant(fam, n, _ptr(s_), _ptr(o_), _ptr(e_), _ptr(a_), int(M), int(alpha[0]),
+                            int(alpha[1]), int(beta0), int(s_bar), int(tau), int(k), int(window),
+                            int(subroutine), int(per_class_s))
     try:
         sc = np.zeros(8, dtype=np.int64)
         L.kvo_scalars(h, _ptr(sc))

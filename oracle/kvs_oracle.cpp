@@ -28,7 +28,10 @@
 // pinned only by reductions to the paper's cases and by invariants):
 //   * schedules built on estimates (class by estimate, kill-and-carry),
 //   * arrival windows,
-//   * heterogeneous prompt lengths (one scalar s_bar for ladder and k*).
+//   * heterogeneous prompt lengths (one scalar s_bar for ladder and k*),
+//   * the two variants inside the geometric classes (simultaneous batches as the subroutine of a phase -
+//     pinned by 21632 and Example 1's 225, which the batching algorithm must reproduce when one class holds
+//     every job; per-phase prompt length - pinned by the reduction to one prompt length).
 //
 // All quantities are exact integers (int64); nothing here is floating point.
 
@@ -201,14 +204,25 @@ i64 run_slice(Schedule& S, const std::vector<i64>& part, const int32_t* s, const
   return base + last + tau;
 }
 
+// Variants inside the geometric classes (used only by the two geometric families):
+//   subroutine = 1: every phase runs the simultaneous schedule instead of Procedure
+//     StaggeredPipelineSchedule - batches of B_p = floor(M / (s_p + tau_p)) jobs start together every
+//     tau_p rounds (Section "Subroutine: Staggered-Pipeline-Schedule", paragraph "The Simultaneous
+//     Batching Trap"; Appendix "Lower Bounds for SimS"): the comparison the paper argues, inside the
+//     same classes.
+//   per_class = 1: the prompt length that sizes a phase's parallelism is the largest prompt length
+//     among that phase's participants, s_p, instead of the one value s_bar for the whole instance
+//     (the paper has a single prompt length, so both coincide there); the ladder still ends at
+//     M - s_bar.  Peak(k, tau, s_p) <= M keeps the phase feasible since no participant has a longer prompt.
 Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int32_t* o_est,
                 const i64* arrival, i64 M, int a, int b, i64 beta0, i64 s_bar_in, i64 tau_in,
-                i64 k_in, i64 window) {
+                i64 k_in, i64 window, int subroutine = 0, int per_class = 0) {
   Schedule* S = new Schedule();
   S->n = n;
   S->job_start.assign(n, -1);
   S->job_completion.assign(n, -1);
-  if (family < 0 || family > 3 || n < 0 || M < 1 || window < 0 || tau_in < 0 || k_in < 0) {
+  if (family < 0 || family > 3 || n < 0 || M < 1 || window < 0 || tau_in < 0 || k_in < 0 ||
+      subroutine < 0 || subroutine > 1 || per_class < 0 || per_class > 1) {
     S->status = 3; return S;
   }
   i64 s_bar = s_bar_in;
@@ -230,7 +244,7 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
   if (geometric) {
     if (a <= b || b < 1) { S->status = 3; return S; }
     S->tau = ladder(X, a, b, beta0);
-    for (i64 t : S->tau) S->k.push_back(kstar(t, s_bar, M));
+    for (i64 t : S->tau) S->k.push_back(subroutine ? M / (s_bar + t) : kstar(t, s_bar, M));
     S->n_part.assign(S->tau.size(), 0);
   }
 
@@ -267,15 +281,22 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
       std::vector<char> entered(hi - lo, family == FAM_GSA ? 1 : 0), done(hi - lo, 0);
       i64 left = hi - lo;
       for (size_t p = 0; p < S->tau.size() && left > 0; ++p) {
-        const i64 tau = S->tau[p], k = S->k[p];
+        const i64 tau = S->tau[p];
+        i64 k = S->k[p];
         std::vector<i64> part;
         for (i64 i : order) {
           if (!entered[i - lo] && std::min<i64>(std::max<i64>(key(i), 1), X) <= tau) entered[i - lo] = 1;
           if (entered[i - lo] && !done[i - lo]) part.push_back(i);
         }
         S->n_part[p] += static_cast<i64>(part.size());
+        if (per_class && !part.empty()) {
+          i64 s_p = 0;
+          for (i64 i : part) s_p = std::max<i64>(s_p, s[i]);
+          k = subroutine ? M / (s_p + tau) : kstar(tau, s_p, M);
+          S->k[p] = k;                       // of the last window in which the phase has participants
+        }
         if (k < 1) { S->status = 1; return S; }
-        base = run_slice(*S, part, s, o, base, tau, k, static_cast<i64>(p), false);
+        base = run_slice(*S, part, s, o, base, tau, k, static_cast<i64>(p), subroutine != 0);
         for (i64 i : part) if (o[i] <= tau) { done[i - lo] = 1; --left; }
       }
     } else {
@@ -320,6 +341,13 @@ void* kvo_build(int32_t family, int64_t n, const int32_t* s, const int32_t* o, c
                 const int64_t* arrival, int64_t M, int32_t alpha_num, int32_t alpha_den,
                 int64_t beta0, int64_t s_bar, int64_t tau, int64_t k, int64_t window) {
   return build(family, n, s, o, o_est, arrival, M, alpha_num, alpha_den, beta0, s_bar, tau, k, window);
+}
+// The same with the two variants inside the geometric classes (see `build`).
+void* kvo_build_variant(int32_t family, int64_t n, const int32_t* s, const int32_t* o, const int32_t* o_est,
+                        const int64_t* arrival, int64_t M, int32_t alpha_num, int32_t alpha_den,
+                        int64_t beta0, int64_t s_bar, int64_t tau, int64_t k, int64_t window,
+                        int32_t subroutine, int32_t per_class) {
+  return build(family, n, s, o, o_est, arrival, M, alpha_num, alpha_den, beta0, s_bar, tau, k, window, subroutine, per_class);
 }
 void kvo_free(void* h) { delete static_cast<Schedule*>(h); }
 

@@ -425,3 +425,61 @@ def test_bounds_hold_for_schedules_and_optimum():
         B = oracle.bounds(s, o, M, beta0=b0)
         assert oracle.build_schedule("GBA", s, o, M, beta0=b0).flow <= B.upper_gba
         assert oracle.build_schedule("GSA", s, o, M, beta0=b0).flow <= B.upper_gsa
+
+
+# ---- variants inside the geometric classes ------------------------------------------------------
+
+def test_simultaneous_subroutine_reproduces_the_paper_numbers():
+    """With simultaneous batches as the subroutine of every phase, the batching algorithm on an instance
+    whose jobs all fall into one class IS the simultaneous schedule of that class.  Uniform experiment
+    (n = 200, o = 16, s = 0, M = 256, alpha = 2): class tau = 16, B = 256 / 16 = 16, the simultaneous number
+    21632 of the paper's figure.  Example 1 (15 jobs, s = 0, o = 5, M = 15) with the initial slice set to 5:
+    B = 3, flow 225 and the per-round memory 3, 6, 9, 12, 15 repeated."""
+    S = oracle.build_schedule("GBA", [0] * 200, [16] * 200, 256, subroutine=1)
+    assert S.status == 0 and S.flow == 21632
+    assert oracle.build_schedule("GBA", [0] * 200, [16] * 200, 256).flow == 14083       # and staggered: the paper's GBA number
+    S = oracle.build_schedule("GBA", [0] * 15, [5] * 15, 15, beta0=5, subroutine=1)
+    assert S.flow == 225 and int(S.k[0]) == 3
+    assert list(_dense(S).profile) == [3, 6, 9, 12, 15] * 5
+    T = oracle.build_schedule("SIMS", [0] * 15, [5] * 15, 15)
+    assert np.array_equal(S.run_start, T.run_start) and np.array_equal(S.job_completion, T.job_completion)
+    # the slicing algorithm too: every phase is one simultaneous schedule of the remaining jobs
+    G = oracle.build_schedule("GSA", [0] * 15, [5] * 15, 15, beta0=5, subroutine=1)
+    assert G.flow == 225
+
+
+def test_class_variants_invariants_and_reductions():
+    rng = np.random.default_rng(77)
+    for alpha in [(2, 1), (3, 2)]:
+        for it in range(80):
+            s, o, M = _random_instance(rng, hetero=it % 2 == 0)
+            for fam in ("GBA", "GSA"):
+                base = oracle.build_schedule(fam, s, o, M, alpha=alpha)
+                for sub in (0, 1):
+                    for pc in (0, 1):
+                        S = oracle.build_schedule(fam, s, o, M, alpha=alpha, subroutine=sub, per_class_s=pc)
+                        assert S.status == 0 and S.n_unfinished == 0
+                        assert _dense(S).peak <= M                                   # every round fits
+                        assert np.array_equal(S.job_completion, S.job_start + o)
+                        # inside a phase: rank r starts floor(r tau / k) (staggered) or floor(r / k) tau (batches)
+                        b0 = 0
+                        for p in range(len(S.tau)):
+                            sel = S.run_phase == p
+                            N = int(sel.sum())
+                            if N == 0:
+                                continue
+                            tau = int(S.tau[p])
+                            st = S.run_start[sel]
+                            kk = int(S.k[p])
+                            r = np.arange(N)
+                            assert np.array_equal(st, b0 + ((r // kk) * tau if sub else (r * tau) // kk))
+                            b0 = int(st[-1]) + tau
+                            s_p = int(max(s[S.run_job[sel]])) if pc else int(S.s_bar)
+                            assert kk == (M // (s_p + tau) if sub else oracle.kstar(tau, s_p, M))
+                    # one prompt length: the per-phase value is that length, nothing changes
+                    if it % 2 == 1:
+                        assert _same(oracle.build_schedule(fam, s, o, M, alpha=alpha, per_class_s=1), base)
+                # a shorter prompt bound can only raise the parallelism: no job starts later
+                P = oracle.build_schedule(fam, s, o, M, alpha=alpha, per_class_s=1)
+                assert np.all(P.job_start <= base.job_start) and P.flow <= base.flow
+    assert oracle.build_schedule("GBA", [1], [1], 10, subroutine=2).status == 3
