@@ -120,6 +120,13 @@ typedef struct {
   int64_t tau;                  /* SPS/SIMS slice length; 0 = largest key of the (sub-)instance */
   int64_t k;                    /* SPS: parallelism, 0 = k*(tau, s_bar) (Eq. max-parallelism);
                                    SIMS: batch size, 0 = floor(M / (s_bar + tau)) */
+  /* Variants inside the geometric classes (GBA / GSA only; both 0 = the paper's algorithms). */
+  int32_t subroutine;           /* 0: every phase runs Procedure StaggeredPipelineSchedule; 1: every phase runs the
+                                   simultaneous schedule instead - batches of floor(M / (s + tau_p)) jobs start together
+                                   every tau_p rounds (Section "Subroutine: Staggered-Pipeline-Schedule", paragraph "The
+                                   Simultaneous Batching Trap"; Appendix "Lower Bounds for SimS") */
+  int32_t per_class_s;          /* 1: the prompt length that sizes a phase's parallelism (or batch) is the longest prompt
+                                   among that phase's participants instead of s_bar; the ladder still ends at M - s_bar */
 } kvs_setting;
 
 /* Per-job and per-run outputs of the builder.  Any pointer may be NULL to skip that output. */
@@ -259,7 +266,14 @@ typedef struct {
   const int64_t* k;             /* HOST [n_k], each in [1, 2^31) */
   int32_t n_tau;
   int32_t n_k;                  /* n_tau * n_k <= 65536 */
-  int32_t family;               /* KVS_SPS or KVS_SIMS */
+  int32_t family;               /* KVS_SPS or KVS_SIMS: the (tau, k) grid; KVS_GBA or KVS_GSA: the beta0 grid below */
+  /* Geometric families: the initial slice of the ladder is a tunable parameter (footnote to the overview of
+   * the slicing algorithm; the experiments use 64 and 256).  One evaluation per entry of beta0 (0 = the
+   * paper's (M - s_bar) / alpha^ell); tau, k, n_tau, n_k are ignored and every output has n_beta0 entries. */
+  int32_t n_beta0;              /* <= 65536 */
+  const int64_t* beta0;         /* HOST [n_beta0], each in [0, 2^31) */
+  int32_t alpha_num, alpha_den;
+  int32_t subroutine, per_class_s;   /* as in kvs_setting */
 } kvs_sweep_params;
 
 typedef struct {                /* DEVICE, each [n_tau * n_k], tau-major; any may be NULL */
@@ -271,7 +285,10 @@ typedef struct {                /* DEVICE, each [n_tau * n_k], tau-major; any ma
   uint8_t* feasible;            /* peak <= M */
 } kvs_sweep_out;
 
-/* For each (tau, k): job with rank r (stable order by exact response length) starts at
+/* Geometric families: for each beta0 the schedule of kvs_evaluate_built with s_bar = the longest prompt;
+ * n_completed = jobs that complete (all of them unless the evaluation is infeasible: then peak = -1,
+ * feasible = 0 and n_completed = 0).  The instances must be offline and carry no estimates.
+ * For each (tau, k): job with rank r (stable order by exact response length) starts at
  * floor(r*tau/k) (SPS, Procedure StaggeredPipelineSchedule) or floor(r/k)*tau (SIMS), runs
  * min(o, tau) rounds and completes iff o <= tau; reports flow over completed jobs, their count,
  * the exact peak of the memory profile (Eq. Memory-Feasibility), horizon and job-steps.

@@ -143,6 +143,20 @@ class Scheduler:
         ctx.bounds(inst, settings, out, max_jobs=max_n)
         return out
 
+    def sweep_beta0(self, inst: Instances, instance: int, family, M: int, beta0, alpha=(2, 1), subroutine=0,
+                    per_class_s=0) -> dict:
+        """GBA / GSA over a list of initial slices on one instance; returns device tensors [n_beta0]."""
+        dev = inst.s.device
+        N, I, max_n, _ = self._sizes(inst)
+        n_set = len(beta0)
+        ctx = self.context(binding.workspace_bytes(N, I, max_n, n_set))
+        out = {f: torch.zeros(n_set, dtype=torch.int64, device=dev)
+               for f in ("peak", "flow", "n_completed", "horizon", "job_steps")}
+        out["feasible"] = torch.zeros(n_set, dtype=torch.uint8, device=dev)
+        ctx.sweep(inst, instance, family, M, [], [], out, max_jobs=max_n, beta0=beta0, alpha=alpha,
+                  subroutine=subroutine, per_class_s=per_class_s)
+        return out
+
     def sweep(self, inst: Instances, instance: int, family, M: int, tau, k) -> dict:
         """SPS / SimS over a (tau, k) grid on one instance; returns device tensors [n_tau, n_k]."""
         dev = inst.s.device

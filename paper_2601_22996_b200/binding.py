@@ -22,7 +22,8 @@ FAMILY = {"GBA": GBA, "GSA": GSA, "SPS": SPS, "SIMS": SIMS}
 EVAL_OK, EVAL_INFEASIBLE, EVAL_RANGE, EVAL_CAPACITY, EVAL_BAD_INPUT = 0, 1, 2, 4, 8
 
 SETTING_DTYPE = np.dtype([("instance", "<i8"), ("family", "<i4"), ("alpha_num", "<i4"), ("alpha_den", "<i4"),
-                          ("s_bar", "<i4"), ("M", "<i8"), ("beta0", "<i8"), ("tau", "<i8"), ("k", "<i8")],
+                          ("s_bar", "<i4"), ("M", "<i8"), ("beta0", "<i8"), ("tau", "<i8"), ("k", "<i8"),
+                          ("subroutine", "<i4"), ("per_class_s", "<i4")],
                          align=True)
 
 
@@ -62,7 +63,8 @@ class _Runs(Structure):
 
 class _SweepParams(Structure):
     _fields_ = [("instance", c_int64), ("M", c_int64), ("tau", c_void_p), ("k", c_void_p),
-                ("n_tau", c_int32), ("n_k", c_int32), ("family", c_int32)]
+                ("n_tau", c_int32), ("n_k", c_int32), ("family", c_int32), ("n_beta0", c_int32), ("beta0", c_void_p),
+                ("alpha_num", c_int32), ("alpha_den", c_int32), ("subroutine", c_int32), ("per_class_s", c_int32)]
 
 
 class _SweepOut(Structure):
@@ -129,7 +131,7 @@ def evaluate_schedule_noalloc(runs: dict, ev: dict, capacity_total: int, device:
 
 
 def make_settings(rows) -> np.ndarray:
-    """Settings array from dicts: instance, family, M [, alpha, s_bar, beta0, tau, k]."""
+    """Settings array from dicts: instance, family, M [, alpha, s_bar, beta0, tau, k, subroutine, per_class_s]."""
     out = np.zeros(len(rows), dtype=SETTING_DTYPE)
     for i, r in enumerate(rows):
         fam = r["family"]
@@ -141,10 +143,12 @@ def make_settings(rows) -> np.ndarray:
         out[i]["beta0"] = r.get("beta0", 0)
         out[i]["tau"] = r.get("tau", 0)
         out[i]["k"] = r.get("k", 0)
+        out[i]["subroutine"] = r.get("subroutine", 0)
+        out[i]["per_class_s"] = r.get("per_class_s", 0)
     return out
 
 
-def settings_grid(instances, families, Ms, alpha=(2, 1)) -> np.ndarray:
+def settings_grid(instances, families, Ms, alpha=(2, 1), subroutine=0, per_class_s=0) -> np.ndarray:
     """Vectorised settings: every (instance, M, family) combination, instance-major.
 
     ``Ms`` is either one list shared by all instances or an array [n_instances, n_M]."""
@@ -158,6 +162,9 @@ def settings_grid(instances, families, Ms, alpha=(2, 1)) -> np.ndarray:
     out["M"] = Ms[None, :, None] if Ms.ndim == 1 else Ms[:, :, None]
     out["alpha_num"], out["alpha_den"] = alpha
     out["s_bar"] = -1
+    geo = out["family"] <= GSA
+    out["subroutine"] = np.where(geo, subroutine, 0)
+    out["per_class_s"] = np.where(geo, per_class_s, 0)
     return out.reshape(-1)
 
 
@@ -273,13 +280,17 @@ class Context:
         self._keep = (runs, ev)
         self._check(self._lib.kvs_evaluate_schedule(self._ctx, ctypes.byref(cr), ctypes.byref(eo)))
 
-    def sweep(self, inst: Instances, instance: int, family, M: int, tau, k, out: dict, max_jobs: int | None = None):
-        """kvs_sweep over the grid tau x k (host lists); ``out`` maps field names to CUDA tensors."""
+    def sweep(self, inst: Instances, instance: int, family, M: int, tau, k, out: dict, max_jobs: int | None = None,
+              beta0=(), alpha=(2, 1), subroutine=0, per_class_s=0):
+        """kvs_sweep over the grid tau x k (SPS / SIMS) or over the initial slices beta0 (GBA / GSA); host lists;
+        ``out`` maps field names to CUDA tensors."""
         ci = self._instances(inst, 0, max_jobs)
         tau = np.ascontiguousarray(tau, dtype=np.int64)
         k = np.ascontiguousarray(k, dtype=np.int64)
+        b0 = np.ascontiguousarray(beta0, dtype=np.int64)
         fam = FAMILY[family] if isinstance(family, str) else family
-        sp = _SweepParams(instance, M, tau.ctypes.data_as(c_void_p), k.ctypes.data_as(c_void_p), tau.size, k.size, fam)
+        sp = _SweepParams(instance, M, tau.ctypes.data_as(c_void_p), k.ctypes.data_as(c_void_p), tau.size, k.size, fam,
+                          b0.size, b0.ctypes.data_as(c_void_p), alpha[0], alpha[1], subroutine, per_class_s)
         so = _SweepOut(*[_p(out.get(f[0])) for f in _SweepOut._fields_])
-        self._keep = (tau, k, inst, out)
+        self._keep = (tau, k, b0, inst, out)
         self._check(self._lib.kvs_sweep(self._ctx, ctypes.byref(ci), ctypes.byref(sp), ctypes.byref(so)))

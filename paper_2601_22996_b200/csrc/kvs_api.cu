@@ -51,6 +51,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // is a prefix of the layout with staging.
 struct Layout {
   size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter, slow_list, walk_list, light_list;
+  size_t sweep_unf, sweep_stat;                                         // unfinished counts and status words of a sweep over initial slices
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
   size_t total;
@@ -76,6 +77,8 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.slow_list = take(static_cast<size_t>(P) * 8);
   L.walk_list = take(static_cast<size_t>(P) * 8);
   L.light_list = take(static_cast<size_t>(P) * 8);
+  L.sweep_unf = take(static_cast<size_t>(P) * 8);
+  L.sweep_stat = take(static_cast<size_t>(P) * 4);
   if (staging) {
     L.st_off = take(static_cast<size_t>(I + 1) * 8);
     L.st_s = take(static_cast<size_t>(N) * 4);
@@ -159,6 +162,10 @@ int check_settings(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* s
     if (s.s_bar < -1) return fail(ctx, KVS_E_ARG, "settings: s_bar < -1");
     if (s.tau < 0 || s.tau >= KVS_TIME_LIMIT || s.k < 0 || s.k >= KVS_TIME_LIMIT)
       return fail(ctx, KVS_E_RANGE, "settings: tau or k outside [0, 2^31)");
+    if (s.subroutine < 0 || s.subroutine > 1 || s.per_class_s < 0 || s.per_class_s > 1)
+      return fail(ctx, KVS_E_ARG, "settings: subroutine and per_class_s are 0 or 1");
+    if ((s.subroutine || s.per_class_s) && s.family != KVS_GBA && s.family != KVS_GSA)
+      return fail(ctx, KVS_E_ARG, "settings: subroutine and per_class_s apply to the geometric families only");
     if (s.family == KVS_GBA || s.family == KVS_GSA) {
       if (s.alpha_den < 1 || s.alpha_num <= s.alpha_den) return fail(ctx, KVS_E_ARG, "settings: alpha must be > 1");
       if (s.beta0 < 0 || s.beta0 >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: beta0 outside [0, 2^31)");
@@ -671,7 +678,34 @@ int kvs_sweep(kvs_ctx* ctx, const kvs_instances* inst, const kvs_sweep_params* p
   if (!params || !out) return fail(ctx, KVS_E_ARG, "sweep: params or out is null");
   if (inst->o_est || inst->window != 0) return fail(ctx, KVS_E_ARG, "sweep: needs offline instances ordered by the exact response length");
   if (params->instance < 0 || params->instance >= inst->n_instances) return fail(ctx, KVS_E_ARG, "sweep: instance out of range");
-  if (params->family != KVS_SPS && params->family != KVS_SIMS) return fail(ctx, KVS_E_ARG, "sweep: family must be SPS or SIMS");
+  if (params->family == KVS_GBA || params->family == KVS_GSA) {
+    // one evaluation per initial slice, through the fused path, scalars only
+    if (params->n_beta0 < 0 || params->n_beta0 > 65536) return fail(ctx, KVS_E_RANGE, "sweep: more than 65536 initial slices");
+    if (params->n_beta0 == 0) return KVS_OK;
+    if (!params->beta0) return fail(ctx, KVS_E_ARG, "sweep: null grid");
+    const int64_t P = params->n_beta0;
+    std::vector<kvs_setting> st(static_cast<size_t>(P));
+    for (int64_t i = 0; i < P; ++i) {
+      kvs_setting& s = st[static_cast<size_t>(i)];
+      s = kvs_setting{};
+      s.instance = params->instance; s.family = params->family; s.alpha_num = params->alpha_num; s.alpha_den = params->alpha_den;
+      s.s_bar = -1; s.M = params->M; s.beta0 = params->beta0[i]; s.subroutine = params->subroutine; s.per_class_s = params->per_class_s;
+    }
+    const Layout L = make_layout(inst->n_jobs_total, inst->n_instances, inst->max_jobs_per_instance, P, false);
+    if (L.total > ctx->workspace_bytes) return fail(ctx, KVS_E_CAPACITY, "workspace too small for the sweep (see kvs_workspace_bytes)");
+    kvs_eval_out ev{};
+    ev.peak = out->peak; ev.flow = out->flow; ev.horizon = out->horizon; ev.job_steps = out->job_steps; ev.feasible = out->feasible;
+    ev.n_unfinished = reinterpret_cast<int64_t*>(ctx->workspace + L.sweep_unf);
+    ev.status = reinterpret_cast<int32_t*>(ctx->workspace + L.sweep_stat);
+    rc = run_fused(ctx, inst, st.data(), P, nullptr, &ev, 1);
+    if (rc) return rc;
+    if (out->n_completed) {
+      const cudaError_t ce = kvs_launch_completed(inst->job_off + params->instance, ev.n_unfinished, ev.status, out->n_completed, P, ctx->stream);
+      if (ce != cudaSuccess) return fail_cuda(ctx, ce, "sweep launch");
+    }
+    return KVS_OK;
+  }
+  if (params->family != KVS_SPS && params->family != KVS_SIMS) return fail(ctx, KVS_E_ARG, "sweep: unknown family");
   if (params->n_tau < 0 || params->n_k < 0 || static_cast<int64_t>(params->n_tau) * params->n_k > 65536)
     return fail(ctx, KVS_E_RANGE, "sweep: grid larger than 65536 settings");
   if (params->n_tau == 0 || params->n_k == 0) return KVS_OK;

@@ -95,7 +95,14 @@ __device__ __forceinline__ void add_event(u32* dA, u32* dB, int idx, u32 c, u32 
 }
 
 // Geometric ladder by warp 0.  Leaves the number of phases in sh.n_phases (0 = too many).
-__device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_bar, i64 M) {
+// Parallelism of a phase: the largest memory-feasible one of Procedure StaggeredPipelineSchedule (Eq.
+// max-parallelism), or the batch size of the simultaneous schedule; 0 if not even one job fits.
+__device__ __forceinline__ i64 phase_parallelism(i64 tau, i64 s, i64 M, bool batches) {
+  if (s + tau > M) return 0;
+  return batches ? M / (s + tau) : max_parallelism(tau, s, M);
+}
+
+__device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_bar, i64 M, bool batches) {
   const int lane = lane_id();
   if (beta0 <= 0) {
     if (lane == 0) {
@@ -117,7 +124,7 @@ __device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_b
       const int j = L - 1 - p;  // tau_p = floor(X * b^j / a^j)
       const i64 t = (a == 2 && b == 1) ? (X >> j) : static_cast<i64>(static_cast<u128>(X) * sh.pw_b[j] / sh.pw_a[j]);
       sh.tau[p] = t;
-      sh.k[p] = max_parallelism(t, s_bar, M);
+      sh.k[p] = phase_parallelism(t, s_bar, M, batches);
     }
   } else {
     if (lane == 0) {
@@ -129,7 +136,7 @@ __device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_b
         const u128 num = static_cast<u128>(beta0) * pa;
         i64 t = (num >= static_cast<u128>(X) * pb) ? X : static_cast<i64>(num / pb);
         sh.tau[p] = t;
-        sh.k[p] = max_parallelism(t, s_bar, M);
+        sh.k[p] = phase_parallelism(t, s_bar, M, batches);
         if (t >= X) break;
         pa *= static_cast<u128>(a); pb *= static_cast<u128>(b);
       }
@@ -365,6 +372,10 @@ template <bool EVENTS, bool WIDE>
 __device__ __forceinline__ int process_runs_w(const BuildParams& p, Shared& sh, const EvalCtx& ec, const Phase& P,
                                               const int32_t* cur, int32_t* nxt, int C_next, int ra, int rb,
                                               i64 t0, int buf, Acc& acc) {
+  if (P.simultaneous && P.may_carry) {   // simultaneous batches inside the phases of a geometric algorithm with carried jobs
+    if (ec.want_runs) return process_runs_t<true, true, EVENTS, true, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+    return process_runs_t<true, true, EVENTS, false, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
+  }
   if (ec.want_runs) {
     if (P.simultaneous) return process_runs_t<true, false, EVENTS, true, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
     if (P.may_carry) return process_runs_t<false, true, EVENTS, true, WIDE>(p, sh, ec, P, cur, nxt, C_next, ra, rb, t0, buf, acc);
@@ -485,10 +496,9 @@ __device__ __forceinline__ void insert_far_ends(Shared& sh, const EvalCtx& ec, c
 // The phase that completes job j is the later of its key's class and the class of o_j
 // (class(x) = first p with tau_p >= x); its rank there is its position inside the class when no
 // jobs are carried, else the rank noted when it completed.  Also accumulates the flow time.
-__device__ __forceinline__ void write_jobs(const BuildParams& p, const Shared& sh, const EvalCtx& ec, int family,
+__device__ __forceinline__ void write_jobs(const BuildParams& p, const Shared& sh, const EvalCtx& ec, int family, bool simultaneous,
                                            int L, i64 X, int seg_lo, int seg_hi, bool may_carry, Acc& acc) {
   const bool geometric = family == KVS_GBA || family == KVS_GSA;
-  const bool simultaneous = family == KVS_SIMS;
   for (int j = seg_lo + threadIdx.x; j < seg_hi; j += T) {
     const int oj = __ldg(ec.O_JOB + j);
     const int pos = ec.IPERM ? __ldg(ec.IPERM + j) : j;
@@ -559,7 +569,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_e
     const i64 X = M - s_bar;
     const int family = st.family;
     const bool geometric = family == KVS_GBA || family == KVS_GSA;
-    const bool simultaneous = family == KVS_SIMS;
+    // variants inside the geometric classes: simultaneous batches as the subroutine of every phase; the
+    // parallelism of a phase sized by the longest prompt among its participants
+    const bool simultaneous = family == KVS_SIMS || (geometric && st.subroutine == 1);
+    const bool per_class = geometric && st.per_class_s == 1;
     const bool keyed = !(family == KVS_GSA && p.key == nullptr);  // plain GSA keeps the index order
     const int32_t* const KEY = p.key ? p.sorted_key + lo : p.sorted_o + lo;
 
@@ -584,7 +597,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_e
     int status = stats.flags;
     if (!status && (X < 1 || stats.o_max > X)) status = KVS_EVAL_INFEASIBLE;
     if (!status && geometric) {
-      if (tid < 32) build_ladder(sh, X, st.alpha_num, st.alpha_den, st.beta0, s_bar, M);
+      if (tid < 32) build_ladder(sh, X, st.alpha_num, st.alpha_den, st.beta0, s_bar, M, simultaneous);
       __syncthreads();
       if (sh.n_phases == 0) status = KVS_EVAL_RANGE;
     }
@@ -648,6 +661,19 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_e
         Phase P;
         if (tid == 0) sh.pbase[ph] = base;   // read by write_jobs after the window's last barrier
         P.base = base; P.tau = sh.tau[ph]; P.k = sh.k[ph];
+        if (per_class) {
+          // longest prompt among this phase's participants: the carried jobs and the entrants
+          i64 s_p = 0;
+          for (int r = tid; r < N; r += T) {
+            const int pos = r < C ? cur[r] : ent_lo + (r - C);
+            s_p = max_i64(s_p, __ldg(ec.S + seg_lo + pos));
+          }
+          s_p = block_max(s_p, sh.red64, static_cast<i64>(0));
+          P.k = phase_parallelism(P.tau, s_p, M, simultaneous);
+          __syncthreads();                   // every thread has read the old entry
+          if (tid == 0) sh.k[ph] = P.k;      // read by write_jobs after the window's last barrier
+        }
+        if (P.k < 1) { status = KVS_EVAL_INFEASIBLE; break; }
         P.N = N; P.C = C; P.ent_lo = ent_lo; P.ph = ph; P.seg_lo = seg_lo;
         P.simultaneous = simultaneous; P.geometric = geometric;
         P.may_carry = geometric && (family == KVS_GSA || p.key != nullptr);
@@ -729,7 +755,8 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_e
         C = C_next;
         if (C == 0 && ent_hi == nseg) break;   // nothing left in this window
       }
-      write_jobs(p, sh, ec, family, L, X, seg_lo, seg_hi, geometric && (family == KVS_GSA || p.key != nullptr), acc);
+      if (status & KVS_EVAL_INFEASIBLE) break;
+      write_jobs(p, sh, ec, family, simultaneous, L, X, seg_lo, seg_hi, geometric && (family == KVS_GSA || p.key != nullptr), acc);
       seg_lo = seg_hi;
     }
 

@@ -836,6 +836,11 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
     const bool carry = geometric && (family == KVS_GSA || est);
     const bool est_class = est && family == KVS_GBA;          // classes by the clipped estimate
     const bool pow2 = geometric && st.alpha_num == 2 && st.alpha_den == 1 && st.beta0 <= 0;
+    if (geometric && (st.subroutine | st.per_class_s)) {
+      // the variants inside the geometric classes are the general kernel's
+      if (tid == 0) p.slow_list[atomicAdd(p.slow_count, 1ull)] = e;
+      continue;
+    }
     // arrays in schedule order (of the instance)
     const int32_t* const S_ord = (keyed ? p.sorted_s : p.s) + lo;
     const int32_t* const O_ord = (keyed ? p.sorted_o : p.o) + lo;

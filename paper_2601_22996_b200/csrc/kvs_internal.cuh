@@ -132,6 +132,8 @@ cudaError_t kvs_launch_bounds(const i64* job_off, const int32_t* o, const InstSt
 cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,
                               i64* prefix_o, cudaStream_t stream);
 cudaError_t kvs_launch_sweep(const SweepParams& p, i64* acc_peak, u64* acc_flow, cudaStream_t stream);
+// n_completed[i] = (job_off[1] - job_off[0]) - n_unfinished[i] where status[i] has neither the infeasible nor the bad-input bit, else 0
+cudaError_t kvs_launch_completed(const i64* job_off, const i64* n_unfinished, const int32_t* status, i64* n_completed, i64 P, cudaStream_t stream);
 
 // ---- small device helpers ---------------------------------------------------------------------
 #ifdef __CUDACC__

@@ -110,3 +110,18 @@ cudaError_t kvs_launch_sweep(const SweepParams& p, i64* acc_peak, u64* acc_flow,
   k_sweep_finish<<<static_cast<unsigned>((n_set + 255) / 256), 256, 0, stream>>>(p, acc_peak, acc_flow);
   return cudaGetLastError();
 }
+
+namespace {
+__global__ void k_completed(const i64* job_off, const i64* n_unfinished, const int32_t* status, i64* n_completed, i64 P) {
+  const i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= P) return;
+  const bool skipped = (status[i] & (KVS_EVAL_INFEASIBLE | KVS_EVAL_BAD_INPUT)) != 0;
+  n_completed[i] = skipped ? 0 : (job_off[1] - job_off[0]) - n_unfinished[i];
+}
+}  // namespace
+
+cudaError_t kvs_launch_completed(const i64* job_off, const i64* n_unfinished, const int32_t* status, i64* n_completed, i64 P, cudaStream_t stream) {
+  if (P <= 0) return cudaSuccess;
+  k_completed<<<static_cast<unsigned>((P + 255) / 256), 256, 0, stream>>>(job_off, n_unfinished, status, n_completed, P);
+  return cudaGetLastError();
+}

@@ -34,7 +34,8 @@ def check_evaluation(task: dict):
     arr = task.get("arrival") if window else None
     S = oracle.build_schedule(int(st["family"]), task["s"], task["o"], int(st["M"]), o_est=task.get("est"), arrival=arr,
                               alpha=(int(st["alpha_num"]), int(st["alpha_den"])), beta0=int(st["beta0"]),
-                              s_bar=int(st["s_bar"]), tau=int(st["tau"]), k=int(st["k"]), window=window)
+                              s_bar=int(st["s_bar"]), tau=int(st["tau"]), k=int(st["k"]), window=window,
+                              subroutine=int(st.get("subroutine", 0)), per_class_s=int(st.get("per_class_s", 0)))
     if S.status != 0:
         return (0, None) if int(got["status"]) & (1 | 8) else (0, f"{tag}: oracle status {S.status}, GPU status {got['status']}")
     if int(got["status"]) != 0:

@@ -31,7 +31,8 @@ def oracle_eval(inst: Instances, st, window=0):
     arr = None if (inst.arrival is None or window == 0) else inst.arrival[a:b]
     return oracle.build_schedule(int(st["family"]), inst.s[a:b], inst.o[a:b], int(st["M"]), o_est=est, arrival=arr,
                                  alpha=(int(st["alpha_num"]), int(st["alpha_den"])), beta0=int(st["beta0"]),
-                                 s_bar=int(st["s_bar"]), tau=int(st["tau"]), k=int(st["k"]), window=window)
+                                 s_bar=int(st["s_bar"]), tau=int(st["tau"]), k=int(st["k"]), window=window,
+                                 subroutine=int(st["subroutine"]), per_class_s=int(st["per_class_s"]))
 
 
 def check_batch(inst_cpu: Instances, settings: np.ndarray, *, window=0, want_profile=True, want_runs=True,

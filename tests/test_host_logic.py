@@ -25,10 +25,10 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header():
     import ctypes
-    assert binding.SETTING_DTYPE.itemsize == 56
+    assert binding.SETTING_DTYPE.itemsize == 64 and binding.SETTING_DTYPE.fields['subroutine'][1] == 56
     assert ctypes.sizeof(binding._Instances) == 72 and ctypes.sizeof(binding._ScheduleOut) == 96
     assert ctypes.sizeof(binding._EvalOut) == 72 and ctypes.sizeof(binding._Runs) == 56
-    assert ctypes.sizeof(binding._SweepParams) == 48 and ctypes.sizeof(binding._SweepOut) == 48
+    assert ctypes.sizeof(binding._SweepParams) == 72 and binding._SweepParams.beta0.offset == 48 and ctypes.sizeof(binding._SweepOut) == 48
 
 
 def test_no_gpu_means_a_loud_failure():
