@@ -76,7 +76,7 @@ class _BoundsOut(Structure):
     _fields_ = [("upper_gba", c_void_p), ("upper_gsa", c_void_p), ("lower_2m", c_void_p), ("status", c_void_p)]
 
 
-EXPORTS = ["kvs_init", "kvs_destroy", "kvs_last_error", "kvs_set_timing", "kvs_last_timing", "kvs_last_timing_split", "kvs_workspace_bytes",
+EXPORTS = ["kvs_init", "kvs_destroy", "kvs_last_error", "kvs_set_timing", "kvs_last_timing", "kvs_last_timing_split", "kvs_debug_check_word", "kvs_workspace_bytes",
            "kvs_build_schedule", "kvs_evaluate_built", "kvs_evaluate_built_host", "kvs_evaluate_schedule", "kvs_sweep",
            "kvs_evaluate_schedule_noalloc", "kvs_bounds"]
 
@@ -99,6 +99,7 @@ def load(path: str | None = None):
         L.kvs_set_timing.argtypes = [c_void_p, c_int32]
         L.kvs_last_timing.argtypes = [c_void_p, POINTER(c_float), POINTER(c_float)]
         L.kvs_last_timing_split.argtypes = [c_void_p, POINTER(c_float), POINTER(c_float), POINTER(c_float)]
+        L.kvs_debug_check_word.argtypes = [POINTER(c_uint64), POINTER(c_int32), c_int32]
         L.kvs_workspace_bytes.argtypes = [c_int64, c_int64, c_int64, c_int64, c_int64, c_int32, POINTER(c_uint64)]
         L.kvs_build_schedule.argtypes = [c_void_p, POINTER(_Instances), c_void_p, c_int64, POINTER(_ScheduleOut), POINTER(_EvalOut)]
         L.kvs_evaluate_built.argtypes = L.kvs_build_schedule.argtypes
@@ -110,6 +111,15 @@ def load(path: str | None = None):
                                                     ctypes.c_char_p, c_uint64]
         _lib = L
     return _lib
+
+
+def debug_check_word(reset: bool = False) -> tuple[int, bool]:
+    """(first index violation recorded by a checked build, 0 = none; whether the loaded library is a checked build)."""
+    w, c = c_uint64(0), c_int32(0)
+    rc = load().kvs_debug_check_word(ctypes.byref(w), ctypes.byref(c), 1 if reset else 0)
+    if rc:
+        raise KvsError(rc, "kvs_debug_check_word")
+    return int(w.value), bool(c.value)
 
 
 def evaluate_schedule_noalloc(runs: dict, ev: dict, capacity_total: int, device: int | None = None):

@@ -448,6 +448,16 @@ int kvs_last_timing_split(kvs_ctx* ctx, float* sort_ms, float* light_ms, float* 
   return KVS_OK;
 }
 
+int kvs_debug_check_word(uint64_t* word, int32_t* compiled_in, int32_t reset) {
+  unsigned long long w = 0ull;
+  int compiled = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return KVS_E_CUDA;
+  if (kvs_fused_check_word(&w, &compiled, reset) != cudaSuccess) return KVS_E_CUDA;
+  if (word) *word = w;
+  if (compiled_in) *compiled_in = compiled;
+  return KVS_OK;
+}
+
 int kvs_workspace_bytes(int64_t n_jobs_total, int64_t n_instances, int64_t max_jobs_per_instance,
                         int64_t n_evaluations, int64_t generic_capacity, int32_t host_staging, uint64_t* out) {
   if (!out || n_jobs_total < 0 || n_instances < 0 || max_jobs_per_instance < 0 || n_evaluations < 0 || generic_capacity < 0)

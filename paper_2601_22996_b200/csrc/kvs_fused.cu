@@ -44,6 +44,25 @@ constexpr int GCOL = 2049;
 static_assert((TILE & (TILE - 1)) == 0 && ITEMS % 4 == 0 && ITEMS <= 32 && 32 % ITEMS == 0, "tile layout");
 constexpr u32 TIME_LIMIT = 0x7fffffffu - 4u * TILE;   // phase ends stay below this
 
+// Checked build (-DKVS_DEBUG): every computed index into the ring, the per-CTA scratch (class bytes, rank
+// table, lists, start rounds, prefix sums) and the caller's profile and per-job outputs is tested against
+// its bound before the access.  A violation records (code << 56 | index) in one device word - the first
+// one wins - and the access is skipped; nothing traps.  The host reads the word with
+// kvs_debug_check_word.  In the normal build KVS_IN is the constant true and costs nothing.
+#ifdef KVS_DEBUG
+__device__ unsigned long long g_check_word = 0ull;
+__device__ __forceinline__ bool kvs_in_range(i64 idx, i64 limit, int code) {
+  if (idx >= 0 && idx < limit) return true;
+  atomicCAS(&g_check_word, 0ull, (static_cast<ull>(code) << 56) | (static_cast<ull>(idx) & 0x00ffffffffffffffull));
+  return false;
+}
+#define KVS_IN(idx, limit, code) kvs_in_range(static_cast<i64>(idx), static_cast<i64>(limit), (code))
+#else
+#define KVS_IN(idx, limit, code) true
+#endif
+enum { CHK_GCOL = 1, CHK_G = 2, CHK_CLS = 3, CHK_RING = 4, CHK_LIST = 5, CHK_LIST_OUT = 6, CHK_PS = 7, CHK_PROFILE = 8,
+       CHK_JOB_OUT = 11, CHK_FIN = 12, CHK_Z = 13 };
+
 struct FShared {
   u128 pw_a[MAXP + 1];
   u128 pw_b[MAXP + 1];
@@ -89,6 +108,7 @@ __device__ __forceinline__ u32 slot_mul(u32 r, u32 tau, u32 k, u64 kinv) {
 
 // Word of the round `rel` rounds after the origin of ring half `buf`, 0 <= rel < 2*TILE.
 __device__ __forceinline__ int ring(int buf, int rel) {
+  if (!KVS_IN(rel, 2 * TILE, CHK_RING)) rel = 0;
   const int e = (buf * TILE + rel) & (2 * TILE - 1);
   return e + ((e >> 5) << 2);
 }
@@ -105,6 +125,7 @@ struct PhaseView {
   const u32* G;
   const u32* gcol;        // column ph of G in shared memory, or NULL
   int L, ph, nsegs;
+  int cls_cap, g_cap;     // bytes of cls and words of G in this CTA's scratch
   int n_src;              // positions of the window (S and O may be read below this index)
   int x_lo, x_hi;
   u32 tau, k, qt, rt;     // tau = qt*k + rt
@@ -116,7 +137,8 @@ constexpr int SEG = 256;  // positions per warp step: 8 consecutive positions pe
 
 // participants of the phase before segment `seg`
 __device__ __forceinline__ int rank_before(const PhaseView& P, int seg) {
-  return static_cast<int>(P.gcol ? P.gcol[seg] : P.G[seg * P.L + P.ph]);
+  if (P.gcol) return KVS_IN(seg, GCOL, CHK_GCOL) ? static_cast<int>(P.gcol[seg]) : 0;
+  return KVS_IN(seg * P.L + P.ph, P.g_cap, CHK_G) ? static_cast<int>(P.G[seg * P.L + P.ph]) : 0;
 }
 
 // The 8 positions of one lane in segment `seg`: bit j of `bits` is set if position xb + j takes part,
@@ -137,7 +159,7 @@ __device__ __forceinline__ LaneGroup lane_group(const PhaseView& P, int seg) {
   const int lane = lane_id();
   if (FILTER) {
     g.xb = seg * SEG + 8 * lane;
-    const uint2 cw = *reinterpret_cast<const uint2*>(P.cls + g.xb);
+    const uint2 cw = KVS_IN(g.xb + 7, P.cls_cap, CHK_CLS) ? *reinterpret_cast<const uint2*>(P.cls + g.xb) : make_uint2(0, 0);
     const int room = P.x_hi - g.xb;                        // positions of this lane below x_hi
     const u32 lim = room >= 8 ? 0xffu : (room > 0 ? (1u << room) - 1u : 0u);
     const u32 p4 = static_cast<u32>(P.ph) * 0x01010101u;
@@ -469,6 +491,7 @@ struct ListView {
   const uint2* cur;
   int C;
   int src;
+  int cap;                // entries of either list in this CTA's scratch
 };
 
 // Run visit over a list: ranks [ra, rb), one to four consecutive ranks per thread, so that a tile
@@ -497,7 +520,7 @@ __device__ __forceinline__ int visit_list(FShared& sh, const PhaseView& P, const
         on[j] = j < rpt && r < rb;
         s_[j] = 0; o_[j] = 0;
         if (on[j]) {
-          if (r < V.C) { const uint2 e = V.cur[r]; s_[j] = e.x; o_[j] = e.y; }
+          if (r < V.C) { if (KVS_IN(r, V.cap, CHK_LIST)) { const uint2 e = V.cur[r]; s_[j] = e.x; o_[j] = e.y; } }
           else { s_[j] = static_cast<u32>(__ldg(P.S + V.src + (r - V.C))); o_[j] = static_cast<u32>(__ldg(P.O + V.src + (r - V.C))); }
         }
       }
@@ -568,7 +591,7 @@ __device__ __forceinline__ int visit_list(FShared& sh, const PhaseView& P, const
     int off = C_next + block_count_scan(__popc(cmask), sh.red32, &total);
 #pragma unroll
     for (int j = 0; j < RPT; ++j)
-      if (cmask >> j & 1u) nxt[off++] = keep[j];
+      if (cmask >> j & 1u) { if (KVS_IN(off, V.cap, CHK_LIST_OUT)) nxt[off] = keep[j]; ++off; }
     C_next += total;
   }
   return C_next;
@@ -586,7 +609,7 @@ __device__ __forceinline__ void insert_far_ends_list(FShared& sh, const PhaseVie
     if (rr < r_hi) {
       const int r = static_cast<int>(rr);
       u32 si, oi;
-      if (r < V.C) { const uint2 e = V.cur[r]; si = e.x; oi = e.y; }
+      if (r < V.C) { uint2 e = make_uint2(0, 1); if (KVS_IN(r, V.cap, CHK_LIST)) e = V.cur[r]; si = e.x; oi = e.y; }
       else { si = static_cast<u32>(__ldg(P.S + V.src + (r - V.C))); oi = static_cast<u32>(__ldg(P.O + V.src + (r - V.C))); }
       const u32 q = slot32(static_cast<u32>(r), P.tau, P.k);
       const u32 end = q + (oi < P.tau ? oi : P.tau);
@@ -610,7 +633,8 @@ __device__ __forceinline__ void insert_far_ends_list(FShared& sh, const PhaseVie
 // forms the events of its own ITEMS rounds of the tile - starts at u and ends of the runs started
 // at u - tau - and adds them to its own words of the ring: no atomics, no dependence on the number
 // of runs.  u0 = offset of the tile's origin inside the phase.
-__device__ __forceinline__ void pure_phase_events(FShared& sh, const PhaseView& P, const u32* __restrict__ PS, int N, int u0, int buf) {
+__device__ __forceinline__ void pure_phase_events(FShared& sh, const PhaseView& P, const u32* __restrict__ PS, int ps_cap, int N, int u0, int buf) {
+  (void)ps_cap;
   const int e0 = ITEMS * static_cast<int>(threadIdx.x);
   const int w0 = ring(buf, e0);
   const u32 tau = P.tau, k = P.k;
@@ -624,7 +648,7 @@ __device__ __forceinline__ void pure_phase_events(FShared& sh, const PhaseView& 
     i64 u = ufirst - 1;
     if (u >= 0) divmod_u(static_cast<u64>(u + 1) * k, tau, &Q, &R);
     u32 b_prev = u >= 0 ? static_cast<u32>(min(static_cast<u64>(N), Q + (R > 0))) : 0u;
-    u32 ps_prev = PS[b_prev];
+    u32 ps_prev = KVS_IN(b_prev, ps_cap, CHK_PS) ? PS[b_prev] : 0u;
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       ++u;
@@ -634,7 +658,7 @@ __device__ __forceinline__ void pure_phase_events(FShared& sh, const PhaseView& 
       if (u >= 0 && land < static_cast<i64>(P.len)) {
         const u32 b = static_cast<u32>(min(static_cast<u64>(N), Q + (R > 0)));
         if (b != b_prev) {
-          const u32 ps = PS[b];
+          const u32 ps = KVS_IN(b, ps_cap, CHK_PS) ? PS[b] : 0u;
           const u32 cnt = b - b_prev;
           const u32 c = (ps - ps_prev) - cnt * (P.base + static_cast<u32>(u));
           if (stream == 0) { sh.dA[w0 + i] += c; sh.dB[w0 + i] += cnt; }
@@ -750,7 +774,7 @@ __device__ __forceinline__ void scan_tile(FShared& sh, int buf, i64 t0, int wlen
 #pragma unroll
     for (int i = 1; i < ITEMS; ++i) m = max(m, mem[i]);
     peak = max(peak, m);
-    if (prof_cap > 0) {
+    if (prof_cap > 0 && KVS_IN(t0 + e0, prof_cap - (ITEMS - 1), CHK_PROFILE)) {
       int4* dst = reinterpret_cast<int4*>(prof + t0 + e0);
 #pragma unroll
       for (int v = 0; v < VEC; ++v)
@@ -768,13 +792,13 @@ __device__ __forceinline__ void scan_tile(FShared& sh, int buf, i64 t0, int wlen
     for (int v = 0; v < VEC; ++v) {
       const i64 rs = t0 + e0 + 4 * v;
       int32_t* dst = prof + rs;
-      if (rs >= lo && rs + 4 <= hi) {
+      if (rs >= lo && rs + 4 <= hi && KVS_IN(rs, prof_cap - 3, CHK_PROFILE)) {
         *reinterpret_cast<int4*>(dst) = make_int4(static_cast<int>(mem[4 * v]), static_cast<int>(mem[4 * v + 1]),
                                                   static_cast<int>(mem[4 * v + 2]), static_cast<int>(mem[4 * v + 3]));
       } else if (rs + 4 > lo && rs < hi) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          if (rs + i >= lo && rs + i < hi) dst[i] = static_cast<int>(mem[4 * v + i]);
+          if (rs + i >= lo && rs + i < hi && KVS_IN(rs + i, prof_cap, CHK_PROFILE)) dst[i] = static_cast<int>(mem[4 * v + i]);
       }
     }
   }
@@ -806,6 +830,12 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
   uint2* const list0 = reinterpret_cast<uint2*>(reinterpret_cast<unsigned char*>(G) + ((static_cast<size_t>(p.max_jobs) / SEG + 2) * MAXP * 4));
   uint2* const list1 = list0 + (p.max_jobs + 1);
   u32* const fin_start = reinterpret_cast<u32*>(p.fin_rank) + static_cast<i64>(blockIdx.x) * p.max_jobs;
+  // bounds of the scratch parts, for the checked build
+  const int cls_cap = static_cast<int>((p.max_jobs + SEG + 15) & ~static_cast<i64>(15));       // bytes
+  const int g_cap = static_cast<int>((static_cast<size_t>(p.max_jobs) / SEG + 2) * MAXP);       // words
+  const int list_cap = static_cast<int>(p.max_jobs + 1);                                        // (s, o) pairs per list
+  const int z_cap = static_cast<int>(KVS_CTA_SCRATCH(p.max_jobs) / 4);                          // words of the whole block
+  (void)cls_cap; (void)g_cap; (void)list_cap; (void)z_cap;
   if (!LIGHT) {
     for (int i = tid; i < RINGW; i += T) { sh.dA[i] = 0; sh.dB[i] = 0; }
   }
@@ -941,7 +971,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             }
             if (j < 4) w0 |= c << (8 * j); else w1 |= c << (8 * (j - 4));
           }
-          *reinterpret_cast<uint2*>(cls + xb) = make_uint2(w0, w1);
+          if (KVS_IN(xb + 7, cls_cap, CHK_CLS)) *reinterpret_cast<uint2*>(cls + xb) = make_uint2(w0, w1);
           __syncwarp();
           u32 h0 = lane < L ? sh.cnt[warp][lane] : 0u;
           u32 h1 = lane + 32 < L ? sh.cnt[warp][lane + 32] : 0u;
@@ -952,15 +982,17 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
           h2 = warp_suffix(h2);
           h1 = warp_suffix(h1) + __shfl_sync(0xffffffffu, h2, 0);
           h0 = warp_suffix(h0) + __shfl_sync(0xffffffffu, h1, 0);
-          if (lane < L) G[seg * L + lane] = h0;
-          if (lane + 32 < L) G[seg * L + lane + 32] = h1;
-          if (lane + 64 < L) G[seg * L + lane + 64] = h2;
+          if (KVS_IN(seg * L + L - 1, g_cap, CHK_G)) {
+            if (lane < L) G[seg * L + lane] = h0;
+            if (lane + 32 < L) G[seg * L + lane + 32] = h1;
+            if (lane + 64 < L) G[seg * L + lane + 64] = h2;
+          }
           __syncwarp();
         }
         __syncthreads();
         // exclusive sums over the segments; row nsegs = totals
         const int rpw = (nsegs + WARPS - 1) / WARPS;
-        const int sa = min(nsegs, warp * rpw), sb = min(nsegs, sa + rpw);
+        const int sa = min(nsegs, warp * rpw), sb = KVS_IN(nsegs * L + L - 1, g_cap, CHK_G) ? min(nsegs, sa + rpw) : sa;
         u32 a0 = 0, a1 = 0, a2 = 0;
         for (int seg = sa; seg < sb; ++seg) {
           if (lane < L) a0 += G[seg * L + lane];
@@ -976,7 +1008,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
           if (lane + 32 < L) { const u32 t = G[seg * L + lane + 32]; G[seg * L + lane + 32] = r1; r1 += t; }
           if (lane + 64 < L) { const u32 t = G[seg * L + lane + 64]; G[seg * L + lane + 64] = r2; r2 += t; }
         }
-        if (warp == WARPS - 1) {
+        if (warp == WARPS - 1 && KVS_IN(nsegs * L + L - 1, g_cap, CHK_G)) {
           // positions that leave in phase q or later: all of them take part in q once they have entered
           if (lane < L) { G[nsegs * L + lane] = r0; sh.np[lane] = r0; }
           if (lane + 32 < L) { G[nsegs * L + lane + 32] = r1; sh.np[lane + 32] = r1; }
@@ -1059,6 +1091,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             } else {
               ++acc.unfinished;
             }
+            if (!KVS_IN(j, n, CHK_JOB_OUT)) continue;
             if (out_start) __stcs(&out_start[j], start);
             if (out_done) __stcs(&out_done[j], done);
           }
@@ -1082,7 +1115,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
 #pragma unroll
             for (int j = 0; j < 8; ++j) ov_[j] = (lim >> j & 1u) ? static_cast<u32>(__ldg(O_ord + seg_lo + xb + j)) : 0u;
           }
-          const uint2 cw = *reinterpret_cast<const uint2*>(cls + xb);
+          const uint2 cw = KVS_IN(xb + 7, cls_cap, CHK_CLS) ? *reinterpret_cast<const uint2*>(cls + xb) : make_uint2(0, 0);
           // smallest and largest class among the warp's valid positions
           u32 lo4 = 0xffu, hi4 = 0u;
 #pragma unroll
@@ -1107,7 +1140,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
               if (lane >= d) incl += y;
             }
             if (eq) {
-              const u32 before = G[seg * L + q] + incl - cnt;
+              const u32 before = (KVS_IN(seg * L + q, g_cap, CHK_G) ? G[seg * L + q] : 0u) + incl - cnt;
 #pragma unroll
               for (int j = 0; j < 8; ++j)
                 if (eq >> j & 1u) rk_[j] = before + static_cast<u32>(__popc(ge & ((1u << j) - 1u)));
@@ -1132,8 +1165,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
           if (keyed) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              if (lim >> j & 1u) fin_start[seg_lo + xb + j] = st_[j];
+              if ((lim >> j & 1u) && KVS_IN(seg_lo + xb + j, p.max_jobs, CHK_FIN)) fin_start[seg_lo + xb + j] = st_[j];
           } else {
+            if (room > 0 && !KVS_IN(seg_lo + xb + min(room, 8) - 1, n, CHK_JOB_OUT)) continue;
             const bool vec_out = room >= 8 && ((seg_lo + xb) & 3) == 0 &&
                                  ((reinterpret_cast<uintptr_t>(out_start) | reinterpret_cast<uintptr_t>(out_done)) & 15u) == 0;
             u32 dn_[8];
@@ -1171,7 +1205,9 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
           __syncthreads();
           for (int j = seg_lo + tid; j < seg_hi; j += T) {
             const u32 oj = static_cast<u32>(__ldg(O_JOB + j));
-            const u32 stt = fin_start[__ldg(IPERM + j)];
+            const int ip = __ldg(IPERM + j);
+            if (!KVS_IN(ip, p.max_jobs, CHK_FIN) || !KVS_IN(j, n, CHK_JOB_OUT)) continue;
+            const u32 stt = fin_start[ip];
             const u32 done = stt + oj;
             acc.hmax = max(acc.hmax, done);
             acc.flow += static_cast<u64>(static_cast<i64>(done) - (ARR ? __ldg(ARR + j) : 0));
@@ -1249,7 +1285,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             F_run += __shfl_sync(0xffffffffu, wi, 31);
 #pragma unroll
             for (int j = 0; j < ITEMS; ++j)
-              if (r + j <= N) Z[r + j] = ps32[2 * static_cast<size_t>(r + j)] - (off + f[j]);
+              if (r + j <= N && KVS_IN(r + j, z_cap, CHK_Z)) Z[r + j] = ps32[2 * static_cast<size_t>(r + j)] - (off + f[j]);
           }
           __syncthreads();
           for (u32 c0 = 0; c0 < N; c0 += TILE) {
@@ -1262,7 +1298,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
 #pragma unroll
             for (int j = 0; j < ITEMS; ++j) {
               o_[j] = r + j < N ? static_cast<u32>(__ldg(Ow + r + j)) : 0u;
-              z_[j] = r + j < N ? Z[r + j] : 0u;
+              z_[j] = (r + j < N && KVS_IN(r + j, z_cap, CHK_Z)) ? Z[r + j] : 0u;
             }
 #pragma unroll
             for (int j = 0; j < ITEMS; ++j) {
@@ -1270,7 +1306,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
                 const u32 t1 = q + min(o_[j], tau);                       // last round of the run, plus one
                 const u64 x = static_cast<u64>(t1) * k + (tau - 1u);      // b = ranks that start before t1
                 const u32 b = (x >> 32) ? static_cast<u32>(min(static_cast<u64>(N), x / tau)) : min(N, static_cast<u32>(x) / tau);
-                acc.peak = max(acc.peak, Z[b] - z_[j] + (b - (r + j)) * t1);
+                if (KVS_IN(b, z_cap, CHK_Z)) acc.peak = max(acc.peak, Z[b] - z_[j] + (b - (r + j)) * t1);
               }
               rem += rt; q += qt;
               if (rem >= k) { rem -= k; ++q; }
@@ -1288,7 +1324,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
         int n_pure = 0;
         u32* const PS = reinterpret_cast<u32*>(list1);
         if (carry && !est) {
-          while (n_pure + 1 < L && static_cast<int>(G[nsegs * L + n_pure + 1]) == nseg) ++n_pure;
+          while (n_pure + 1 < L && KVS_IN(nsegs * L + n_pure + 1, g_cap, CHK_G) && static_cast<int>(G[nsegs * L + n_pure + 1]) == nseg) ++n_pure;
           if (n_pure > 0) {
             u32 run = 0;
             for (int x0 = 0; x0 <= nseg; x0 += T * 4) {
@@ -1315,7 +1351,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
               const u32 off = run + __shfl_sync(0xffffffffu, wi - w, warp) + (incl - tot);
               run += __shfl_sync(0xffffffffu, wi, 31);
 #pragma unroll
-              for (int j = 0; j < 4; ++j) if (x + j <= nseg) PS[x + j] = off + v[j];
+              for (int j = 0; j < 4; ++j) if (x + j <= nseg && KVS_IN(x + j, 2 * list_cap, CHK_PS)) PS[x + j] = off + v[j];
             }
             __syncthreads();
           }
@@ -1326,9 +1362,11 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
           PhaseView P;
           P.S = S_ord + seg_lo; P.O = O_ord + seg_lo;
           P.cls = cls; P.G = G; P.L = L; P.ph = ph; P.nsegs = nsegs;
+          P.cls_cap = cls_cap; P.g_cap = g_cap;
           P.gcol = nullptr;
           if (carry && nsegs < GCOL) {
-            for (int seg = tid; seg <= nsegs; seg += T) sh.gcol[seg] = G[seg * L + ph];
+            for (int seg = tid; seg <= nsegs; seg += T)
+              if (KVS_IN(seg * L + ph, g_cap, CHK_G)) sh.gcol[seg] = G[seg * L + ph];
             P.gcol = sh.gcol;
             __syncthreads();
           }
@@ -1342,7 +1380,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
           const bool combine = sim && P.k >= 32;
           const bool dense = !sim && P.tau < TILE && P.k >= 4 * P.tau;
           ListView V;
-          V.cur = cur; V.C = C; V.src = sh.ent[ph];
+          V.cur = cur; V.C = C; V.src = sh.ent[ph]; V.cap = list_cap;
           if (carry && !list_mode && 2 * N <= nseg) {
             // from here on the participants are kept as a list in rank order: first this phase's
             for (int seg = warp; seg < nsegs; seg += WARPS) {
@@ -1350,7 +1388,10 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
               int r = g.r_first;
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                if (g.bits >> j & 1u) cur[r++] = make_uint2(static_cast<u32>(__ldg(P.S + g.xb + j)), static_cast<u32>(__ldg(P.O + g.xb + j)));
+                if (g.bits >> j & 1u) {
+                  if (KVS_IN(r, list_cap, CHK_LIST_OUT)) cur[r] = make_uint2(static_cast<u32>(__ldg(P.S + g.xb + j)), static_cast<u32>(__ldg(P.O + g.xb + j)));
+                  ++r;
+                }
             }
             list_mode = true;
             V.C = N;
@@ -1380,7 +1421,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             }
             cq += dq; cr += dr;
             if (cr >= utau) { cr -= utau; ++cq; }
-            if (ph < n_pure) pure_phase_events(sh, P, PS, N, u0, buf);
+            if (ph < n_pure) pure_phase_events(sh, P, PS, 2 * list_cap, N, u0, buf);
             else if (sim) visit_runs<true, false>(sh, P, r_next, r_b, u0, buf, dense, combine);
             else if (list_mode) C_next = visit_list(sh, P, V, nxt, C_next, r_next, r_b, u0, buf, dense);
             else if (carry && P.tau < static_cast<u32>(TILE) && P.k >= 8u * P.tau) visit_runs_sliced(sh, P, r_next, r_b, u0, buf, sh.kinv[ph]);
@@ -1487,4 +1528,20 @@ cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam,
   if (fam == KVS_GBA) return launch<false, KVS_GBA>(p, grid, stream);
   if (fam == KVS_GSA) return launch<false, KVS_GSA>(p, grid, stream);
   return launch<false, KVS_FUSED_ANY>(p, grid, stream);
+}
+
+// First violation recorded by the checked build (0 = none); `compiled` = 1 if this library was built with
+// -DKVS_DEBUG.  `reset` clears the word after reading it.
+cudaError_t kvs_fused_check_word(unsigned long long* word, int* compiled, int reset) {
+#ifdef KVS_DEBUG
+  if (compiled) *compiled = 1;
+  cudaError_t e = cudaMemcpyFromSymbol(word, g_check_word, sizeof(unsigned long long));
+  if (e == cudaSuccess && reset) { const unsigned long long z = 0ull; e = cudaMemcpyToSymbol(g_check_word, &z, sizeof(z)); }
+  return e;
+#else
+  if (compiled) *compiled = 0;
+  *word = 0ull;
+  (void)reset;
+  return cudaSuccess;
+#endif
 }

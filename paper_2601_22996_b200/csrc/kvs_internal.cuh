@@ -126,6 +126,7 @@ int kvs_build_ctas_per_sm();
 enum { KVS_FUSED_ANY = -1 };   // instantiation of the fast kernel for any family; the others are named by the family id
 cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam, cudaStream_t stream);
 int kvs_fused_ctas_per_sm(int light);
+cudaError_t kvs_fused_check_word(unsigned long long* word, int* compiled, int reset);
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_bounds(const i64* job_off, const int32_t* o, const InstStats* stats, const kvs_setting* settings,
                               i64 P, const kvs_bounds_out& out, int grid, cudaStream_t stream);
