@@ -29,6 +29,9 @@
 //   * schedules built on estimates (class by estimate, kill-and-carry),
 //   * arrival windows,
 //   * heterogeneous prompt lengths (one scalar s_bar for ladder and k*),
+//   * the dynamic refill of the batching schedule (the paper gives its rule in words; the reading is stated at
+//     `dynamic_refill`; pinned by what the paper promises - no job starts later than in the batching schedule,
+//     every round fits - by a hand-worked instance and by the brute-force optimum as a lower bound),
 //   * the two variants inside the geometric classes (simultaneous batches as the subroutine of a phase -
 //     pinned by 21632 and Example 1's 225, which the batching algorithm must reproduce when one class holds
 //     every job; per-phase prompt length - pinned by the reduction to one prompt length).
@@ -169,7 +172,7 @@ std::vector<i64> ladder(i64 X, int a, int b, i64 beta0) {
   return tau;
 }
 
-enum { FAM_GBA = 0, FAM_GSA = 1, FAM_SPS = 2, FAM_SIMS = 3 };
+enum { FAM_GBA = 0, FAM_GSA = 1, FAM_SPS = 2, FAM_SIMS = 3, FAM_GBAD = 4 };
 
 struct Run { i64 job, phase, start, len, s; };
 
@@ -214,6 +217,41 @@ i64 run_slice(Schedule& S, const std::vector<i64>& part, const int32_t* s, const
 //     among that phase's participants, s_p, instead of the one value s_bar for the whole instance
 //     (the paper has a single prompt length, so both coincide there); the ladder still ends at
 //     M - s_bar.  Peak(k, tau, s_p) <= M keeps the phase feasible since no participant has a longer prompt.
+// Dynamic refill of a batching schedule (Numerical Experiments, "Dynamic Refill (GBA-D)": a job is admitted
+// as soon as the pipeline can go on with it without violating memory feasibility; no job is delayed
+// relative to the baseline schedule, only idle time is filled).  The paper states the rule in words; the
+// reading taken here keeps its two promises by construction:
+//   the plan starts as the batching schedule (every job at its start there, one run per job, no kills);
+//   the jobs are taken in the schedule's order (class by class, shortest first); job i moves to the earliest
+//   round t with d_(i-1) <= t <= g_i (its start in the batching schedule; admissions keep their order) at
+//   which the whole plan - earlier jobs at their new starts, job i at t, later jobs still at their starts in
+//   the batching schedule - fits the budget in every round; t = g_i always qualifies when the batching
+//   schedule itself fits, and is kept otherwise.
+// The check is the definition: add the job's ramp s + u + 1 round by round on top of the plan's memory.
+void dynamic_refill(Schedule& S, i64 M) {
+  i64 T = 0;
+  for (const Run& r : S.runs) T = std::max(T, r.start + r.len);
+  std::vector<i64> mem(static_cast<size_t>(T), 0);
+  for (const Run& r : S.runs)
+    for (i64 u = 0; u < r.len; ++u) mem[r.start + u] += r.s + u + 1;
+  i64 prev = 0;
+  for (Run& r : S.runs) {                       // runs are in (phase, rank) order: the order of admission
+    const i64 g = r.start;
+    for (i64 u = 0; u < r.len; ++u) mem[g + u] -= r.s + u + 1;
+    i64 d = g;
+    for (i64 t = prev; t < g; ++t) {
+      bool fits = true;
+      for (i64 u = 0; u < r.len && fits; ++u) fits = mem[t + u] + r.s + u + 1 <= M;
+      if (fits) { d = t; break; }
+    }
+    for (i64 u = 0; u < r.len; ++u) mem[d + u] += r.s + u + 1;
+    r.start = d;
+    S.job_start[r.job] = d;
+    S.job_completion[r.job] = d + r.len;       // every run of a batching schedule on exact lengths completes its job
+    prev = d;
+  }
+}
+
 Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int32_t* o_est,
                 const i64* arrival, i64 M, int a, int b, i64 beta0, i64 s_bar_in, i64 tau_in,
                 i64 k_in, i64 window, int subroutine = 0, int per_class = 0) {
@@ -221,6 +259,12 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
   S->n = n;
   S->job_start.assign(n, -1);
   S->job_completion.assign(n, -1);
+  bool refill = false;
+  if (family == FAM_GBAD) {
+    if (o_est || window != 0 || subroutine != 0) { S->status = 3; return S; }   // the refill is defined on the plain batching schedule
+    family = FAM_GBA;
+    refill = true;
+  }
   if (family < 0 || family > 3 || n < 0 || M < 1 || window < 0 || tau_in < 0 || k_in < 0 ||
       subroutine < 0 || subroutine > 1 || per_class < 0 || per_class > 1) {
     S->status = 3; return S;
@@ -310,6 +354,7 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
     }
   }
 
+  if (refill && S->status == 0) dynamic_refill(*S, M);
   for (const Run& r : S->runs) {
     S->horizon = std::max(S->horizon, r.start + r.len);
     S->job_steps += r.len;

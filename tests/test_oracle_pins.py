@@ -483,3 +483,47 @@ def test_class_variants_invariants_and_reductions():
                 P = oracle.build_schedule(fam, s, o, M, alpha=alpha, per_class_s=1)
                 assert np.all(P.job_start <= base.job_start) and P.flow <= base.flow
     assert oracle.build_schedule("GBA", [1], [1], 10, subroutine=2).status == 3
+
+
+# ---- dynamic refill of the batching schedule ------------------------------------------------------
+
+def test_dynamic_refill_hand_worked_instance(golden_dir):
+    """M = 10, s = 2, o = 1, 1, 2, 3, 5, 8 (alpha = 2: ladder 1, 2, 4, 8 with k* = 3, 2, 2, 1).  The batching
+    schedule starts the jobs at 0, 0, 1, 3, 7, 15 (flow 46).  Refill, worked by hand from the reading: the job
+    of length 2 fits at 0 beside the two unit jobs (3 + 3 + 3 = 9); the job of length 3 does not fit at 0
+    (9 + 3 > 10) but at 1 (4 + 3, then 4, 5); the job of length 5 fits at 1 too (4 + 3 + 3 = 10, then 4 + 4,
+    5 + 5, 6, 7); the job of length 8 fails at 1 .. 3, fits round 4 but not round 5 from 4 (7 + 4 > 10), and
+    fits from 5 on: starts 0, 0, 0, 1, 1, 5, flow 27, memory 9, 10, 8, 10, 6, 10, 4, 5, ..., 10."""
+    rows = [ln.split() for ln in open(os.path.join(golden_dir, "dynamic_refill_hand_example.txt")) if ln.strip() and not ln.startswith("#")]
+    want = {r[0]: [int(x) for x in r[1:]] for r in rows}
+    S = oracle.build_schedule("GBAD", [2] * 6, want["o"], 10)
+    assert S.status == 0 and list(S.job_start) == want["start"] and S.flow == want["flow"][0]
+    assert list(_dense(S).profile) == want["memory"]
+    assert list(oracle.build_schedule("GBA", [2] * 6, want["o"], 10).job_start) == want["gba_start"]
+
+
+def test_dynamic_refill_keeps_the_paper_promises():
+    """No job starts later than in the batching schedule, admissions keep their order, every round fits, the
+    flow time is at most the batching schedule's (hence within UpperGBA), and at least the optimum."""
+    rng = np.random.default_rng(88)
+    for alpha in [(2, 1), (3, 2), (4, 3)]:
+        for it in range(120):
+            s, o, M = _random_instance(rng, hetero=it % 3 == 0)
+            G = oracle.build_schedule("GBA", s, o, M, alpha=alpha)
+            D = oracle.build_schedule("GBAD", s, o, M, alpha=alpha)
+            assert D.status == 0 and D.n_unfinished == 0 and len(D.run_job) == len(o)
+            assert np.all(D.job_start <= G.job_start) and D.flow <= G.flow
+            assert np.array_equal(D.run_job, G.run_job) and np.all(np.diff(D.run_start) >= 0)
+            assert np.array_equal(D.job_completion, D.job_start + o) and D.job_steps == int(o.sum())
+            assert _dense(D).peak <= M
+            if it % 3:
+                assert D.flow <= oracle.bounds(s, o, M, alpha=alpha).upper_gba
+    for it in range(60):
+        n, s = int(rng.integers(1, 8)), int(rng.integers(0, 6))
+        o = rng.integers(1, 7, n)
+        M = int(s + o.max() + rng.integers(0, 14))
+        assert oracle.opt_bruteforce(s, o, M) <= oracle.build_schedule("GBAD", [s] * n, o, M).flow
+    # a schedule without idle memory cannot move: one job per slot at full length
+    D = oracle.build_schedule("GBAD", [0] * 5, [8] * 5, 8)
+    assert list(D.job_start) == [0, 8, 16, 24, 32]
+    assert oracle.build_schedule("GBAD", [1], [1], 10, window=5).status == 3
