@@ -3,7 +3,7 @@
 path over one batch of seeded synthetic instances).  Prints ONE JSON line on rank 0.
 
     python bench.py --gpus 1 --steps 5 --warmup 3            # config 5, the workload the target is quoted on
-    python bench.py --workload c1|c2|c3|c4|c5|bounds         # the other configs: c4 = the (tau, k) sweep
+    python bench.py --workload c1|c2|c3|c4|c5|c2d|bounds     # the other configs: c4 = the (tau, k) sweep, c2d = dynamic refill
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
     python bench.py --impl reference                         # the CPU oracle, as it stands, on a bounded sample
 """
@@ -34,6 +34,7 @@ WORKLOADS = {
     "c3": ("config3", 256, 100_000, ["GBA", "GSA"], "config 3: 256 instances x 100,000 jobs, online arrivals, estimates, M=2^22"),
     "c4": ("config4", 1, 1_000_000, ["SPS", "SIMS"], "config 4: one instance of 1,000,000 jobs, 64 x 64 (tau, k) grid, SPS and SimS, scalars only"),
     "c5": ("config5", 16_384, 50_000, ["GBA", "GSA", "SPS", "SIMS"], "config 5 (stress): 16,384 instances x 50,000 jobs, mixed distributions, M per instance, four families"),
+    "c2d": ("config2", 1024, 10_000, ["GBAD"], "config 2's instances and budgets under GBA with dynamic refill (GBA-D): batching schedule, then the refill kernel"),
     "bounds": ("config2", 1024, 10_000, ["GBA"], "class-size bounds (kvs_bounds) on config 2's instances and budgets"),
 }
 # The sweep is bound by integer arithmetic on inputs that stay in L2: per candidate round (one per run and

@@ -44,7 +44,16 @@ enum kvs_status {
 /* Schedule families.  GBA: Algorithm "Geometric Batching Algorithm"; GSA: Algorithm
  * "Geometric Slicing Algorithm"; SPS: Procedure "StaggeredPipelineSchedule" run once on the
  * whole instance; SIMS: the simultaneous schedule (Appendix "Lower Bounds for SimS"). */
-enum kvs_family { KVS_GBA = 0, KVS_GSA = 1, KVS_SPS = 2, KVS_SIMS = 3 };
+enum kvs_family { KVS_GBA = 0, KVS_GSA = 1, KVS_SPS = 2, KVS_SIMS = 3,
+                  /* GBA with dynamic refill (Numerical Experiments, "Dynamic Refill (GBA-D)"): the batching schedule is
+                   * formed first; then, in its order, every job moves to the earliest round between the previous
+                   * admission and its own start at which the whole plan - earlier jobs at their new starts, later
+                   * ones still at their old ones - fits the budget in every round.  No job starts later than in the
+                   * batching schedule.  Accepted by kvs_evaluate_built (which needs job_start, job_completion and a
+                   * profile with the batching schedule's horizon as capacity: they are its working storage) and by
+                   * kvs_build_schedule (which reports the batching schedule: its horizon sizes the profile); offline
+                   * instances without estimates only. */
+                  KVS_GBAD = 4 };
 
 /* Bits of the per-evaluation status word. */
 enum kvs_eval_status {

@@ -27,6 +27,7 @@ struct kvs_ctx {
   // host entry point: input copies run on a stream of their own, one event per chunk of instances
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t chunk_ev[KVS_HOST_CHUNKS + 1] = {};
+  std::vector<kvs_setting> settings_tmp;   // a call's settings with the refill family mapped to the batching one
   std::string err;
 };
 
@@ -51,6 +52,7 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 // is a prefix of the layout with staging.
 struct Layout {
   size_t settings, stats, perm, perm_tmp, iperm, sorted_s, sorted_o, sorted_key, prefix_s, lists, fin_rank, counter, slow_list, walk_list, light_list;
+  size_t refill_list;                                                    // evaluations whose batching schedule is refilled afterwards
   size_t sweep_unf, sweep_stat;                                         // unfinished counts and status words of a sweep over initial slices
   size_t st_off, st_s, st_o, st_key, st_arr;                            // host staging (inputs)
   size_t sc_peak, sc_flow, sc_steps, sc_hor, sc_unf, sc_feas, sc_stat;  // host staging (scalars)
@@ -77,6 +79,7 @@ Layout make_layout(int64_t N, int64_t I, int64_t max_n, int64_t P, bool staging)
   L.slow_list = take(static_cast<size_t>(P) * 8);
   L.walk_list = take(static_cast<size_t>(P) * 8);
   L.light_list = take(static_cast<size_t>(P) * 8);
+  L.refill_list = take(static_cast<size_t>(P) * 8);
   L.sweep_unf = take(static_cast<size_t>(P) * 8);
   L.sweep_stat = take(static_cast<size_t>(P) * 4);
   if (staging) {
@@ -157,16 +160,18 @@ int check_settings(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* s
   for (int64_t e = 0; e < P; ++e) {
     const kvs_setting& s = st[e];
     if (s.instance < 0 || s.instance >= inst->n_instances) return fail(ctx, KVS_E_ARG, "settings: instance out of range");
-    if (s.family < KVS_GBA || s.family > KVS_SIMS) return fail(ctx, KVS_E_ARG, "settings: unknown family");
+    if (s.family < KVS_GBA || s.family > KVS_GBAD) return fail(ctx, KVS_E_ARG, "settings: unknown family");
+    if (s.family == KVS_GBAD && (inst->o_est || inst->window != 0 || s.subroutine))
+      return fail(ctx, KVS_E_ARG, "settings: the dynamic refill takes offline instances without estimates and the staggered subroutine");
     if (s.M < 1 || s.M >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: M outside [1, 2^31)");
     if (s.s_bar < -1) return fail(ctx, KVS_E_ARG, "settings: s_bar < -1");
     if (s.tau < 0 || s.tau >= KVS_TIME_LIMIT || s.k < 0 || s.k >= KVS_TIME_LIMIT)
       return fail(ctx, KVS_E_RANGE, "settings: tau or k outside [0, 2^31)");
     if (s.subroutine < 0 || s.subroutine > 1 || s.per_class_s < 0 || s.per_class_s > 1)
       return fail(ctx, KVS_E_ARG, "settings: subroutine and per_class_s are 0 or 1");
-    if ((s.subroutine || s.per_class_s) && s.family != KVS_GBA && s.family != KVS_GSA)
+    if ((s.subroutine || s.per_class_s) && s.family != KVS_GBA && s.family != KVS_GSA && s.family != KVS_GBAD)
       return fail(ctx, KVS_E_ARG, "settings: subroutine and per_class_s apply to the geometric families only");
-    if (s.family == KVS_GBA || s.family == KVS_GSA) {
+    if (s.family == KVS_GBA || s.family == KVS_GSA || s.family == KVS_GBAD) {
       if (s.alpha_den < 1 || s.alpha_num <= s.alpha_den) return fail(ctx, KVS_E_ARG, "settings: alpha must be > 1");
       if (s.beta0 < 0 || s.beta0 >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: beta0 outside [0, 2^31)");
       if (!(s.alpha_num == 2 && s.alpha_den == 1) && !ladder_fits(s.M, s.alpha_num, s.alpha_den))
@@ -199,6 +204,18 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   if (reinterpret_cast<uintptr_t>(v.profile) & 15u) return fail(ctx, KVS_E_ARG, "eval_out: profile must be 16-byte aligned");
   if (!do_profile) v.profile = nullptr;
   if (P == 0) return KVS_OK;
+  // Dynamic refill: the fused kernels form the batching schedule; a last kernel refills it in place.
+  std::vector<int64_t> refill;
+  for (int64_t e = 0; e < P; ++e)
+    if (settings[e].family == KVS_GBAD) refill.push_back(e);
+  if (!refill.empty()) {
+    if (rg) return fail(ctx, KVS_E_ARG, "the host entry point does not take the dynamic refill (it needs per-job results and a profile on the device)");
+    if (do_profile && (!o.job_start || !o.job_completion || !v.profile || o.job_start64 || o.job_completion64 || run_out))
+      return fail(ctx, KVS_E_ARG, "the dynamic refill needs job_start, job_completion and a profile (32-bit, no run list): they are its working storage");
+    ctx->settings_tmp.assign(settings, settings + P);
+    for (int64_t e : refill) ctx->settings_tmp[static_cast<size_t>(e)].family = KVS_GBA;
+    settings = ctx->settings_tmp.data();
+  }
 
   const int64_t N = inst->n_jobs_total, I = inst->n_instances, max_n = inst->max_jobs_per_instance;
   const Layout L = make_layout(N, I, max_n, rg ? rg->P_total : P, false);
@@ -358,6 +375,20 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   bp.counter = counters + 2;
   ce = kvs_launch_build(bp, grid_for(ctx->build_ctas_per_sm), ctx->stream);
   if (ce != cudaSuccess) return fail_cuda(ctx, ce, "build launch");
+  if (do_profile && !refill.empty()) {
+    ce = cudaMemcpyAsync(ws + L.refill_list, refill.data(), refill.size() * 8, cudaMemcpyHostToDevice, ctx->stream);
+    if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of the refill list");
+    RefillParams rp{};
+    rp.job_off = inst->job_off; rp.perm = sp.perm; rp.sorted_s = sp.sorted_s; rp.sorted_o = sp.sorted_o;
+    rp.settings = reinterpret_cast<const kvs_setting*>(settings_dev);
+    rp.eval_list = reinterpret_cast<const i64*>(ws + L.refill_list); rp.n_list = static_cast<i64>(refill.size());
+    rp.job_out_off = o.job_out_off; rp.job_start = o.job_start; rp.job_completion = o.job_completion;
+    rp.profile_off = v.profile_off; rp.profile = v.profile;
+    rp.peak = v.peak; rp.flow = v.flow; rp.horizon = v.horizon; rp.feasible = v.feasible; rp.status = v.status;
+    if (!v.horizon || !v.status) return fail(ctx, KVS_E_ARG, "the dynamic refill needs the horizon and status outputs");
+    ce = kvs_launch_refill(rp, ctx->stream);
+    if (ce != cudaSuccess) return fail_cuda(ctx, ce, "refill launch");
+  }
   if (ctx->timing && !rg) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; ctx->split_timed = fast; }
   return KVS_OK;
 }

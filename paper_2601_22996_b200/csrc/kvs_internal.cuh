@@ -106,6 +106,24 @@ struct GenericParams {
   i64 slots;                // entries of each array; the kernel skips an evaluation whose offsets reach beyond
 };
 
+// Dynamic refill of the batching schedules of the listed evaluations, in place (see kvs_refill.cu).
+struct RefillParams {
+  const i64* job_off;
+  const int32_t* perm;         // key order -> job index, per instance
+  const int32_t* sorted_s;     // prompt and response lengths in key order
+  const int32_t* sorted_o;
+  const kvs_setting* settings;
+  const i64* eval_list;        // evaluations to refill
+  i64 n_list;
+  const i64* job_out_off;
+  int32_t* job_start;          // in: starts of the batching schedule; out: refilled starts
+  int32_t* job_completion;
+  const i64* profile_off;
+  int32_t* profile;            // in: memory of the batching schedule; out: of the refilled one
+  i64* peak; i64* flow; i64* horizon; uint8_t* feasible;
+  const int32_t* status;
+};
+
 struct SweepParams {
   const int32_t* sorted_s;  // the instance in key order
   const int32_t* sorted_o;
@@ -128,6 +146,7 @@ cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam,
 int kvs_fused_ctas_per_sm(int light);
 cudaError_t kvs_fused_check_word(unsigned long long* word, int* compiled, int reset);
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
+cudaError_t kvs_launch_refill(const RefillParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_bounds(const i64* job_off, const int32_t* o, const InstStats* stats, const kvs_setting* settings,
                               i64 P, const kvs_bounds_out& out, int grid, cudaStream_t stream);
 cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,
