@@ -56,9 +56,10 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
-    ap.add_argument("--ncu-traffic", default="", help="csv of `ncu --csv --page raw` with dram__bytes_read.sum / dram__bytes_write.sum of the "
-                                                      "dominant kernel's launches on a small case of this workload")
-    ap.add_argument("--ncu-evals", type=int, default=0, help="evaluations those captured launches processed (traffic is scaled by evaluations)")
+    ap.add_argument("--ncu-traffic", default=os.path.join(ROOT, "profiles", "k_fused_eval_c5_traffic.csv"),
+                    help="csv of `ncu --csv --page raw` with dram__bytes_read.sum / dram__bytes_write.sum of the dominant kernel's launches on a "
+                         "small case of config 5, headed by a line `# evaluations=<n> kvs_fused_sha256=<hash of csrc/kvs_fused.cu at the capture>`; "
+                         "used only while that source file is unchanged")
     return ap.parse_args()
 
 
@@ -180,11 +181,22 @@ def load_peaks():
 
 
 def ncu_traffic(path: str, kernel_substr: str):
-    """dram__bytes_read.sum + dram__bytes_write.sum over the rows of an ncu raw csv whose kernel name contains
-    `kernel_substr`; None if the file is missing or holds no such row."""
+    """(dram__bytes_read.sum + dram__bytes_write.sum over the rows of an ncu raw csv whose kernel name contains
+    `kernel_substr`, evaluations those launches processed), or None if the file is missing, holds no such row, or
+    was captured from another state of the kernel's source."""
+    import hashlib
+    import re
     if not path or not os.path.exists(path):
         return None
     with open(path, newline="") as f:
+        first = f.readline()
+        m = re.match(r"#\s*evaluations=(\d+)\s+kvs_fused_sha256=([0-9a-f]+)", first)
+        if not m:
+            return None
+        with open(os.path.join(ROOT, "paper_2601_22996_b200", "csrc", "kvs_fused.cu"), "rb") as src:
+            if hashlib.sha256(src.read()).hexdigest() != m.group(2):
+                return None                      # the kernel has changed since the counters were taken
+        evals = int(m.group(1))
         rows = [r for r in csv.reader(f) if r]
     head = next((i for i, r in enumerate(rows) if "Kernel Name" in r), None)
     if head is None or head + 2 > len(rows):
@@ -199,7 +211,7 @@ def ncu_traffic(path: str, kernel_substr: str):
             if col in h:
                 total += float(r[h.index(col)].replace(",", "")) * scale.get(units[h.index(col)], 1.0)
                 seen = True
-    return total if seen else None
+    return (total, evals) if seen and evals > 0 else None
 
 
 def run_reference(args):
@@ -491,9 +503,9 @@ def run_fused_workload(args, rank, world, dev, local, dist, binding, Scheduler):
     peak_gbs, peak_kind = load_peaks()
     achieved = alg_bytes / (full_avg * 1e-3) / 1e9 if walked and full_avg > 0 else 0.0
     traffic = None
-    per_launch = ncu_traffic(args.ncu_traffic, "k_fused_eval<0")      # the full variant's launches of the captured small case
-    if per_launch is not None and args.ncu_evals > 0:
-        traffic = per_launch / args.ncu_evals * walked                # traffic grows with the evaluations: each CTA holds one at a time
+    captured = ncu_traffic(args.ncu_traffic, "k_fused_eval<0") if name == "c5" else None   # the full variant's launches of the captured small case
+    if captured is not None:
+        traffic = captured[0] / captured[1] * walked                  # traffic grows with the evaluations: each CTA holds one at a time
     # kernels of one kvs_evaluate_built call: ordering kernel; without estimates one launch of the light
     # variant per SPS / SimS family and one of the full variant per geometric family (with estimates one of
     # each for all families); the full variant for what the light one passes on; the general kernel on the
