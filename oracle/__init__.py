@@ -17,8 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "kvs_oracle.cpp")
 _LIB = os.path.join(_HERE, "libkvs_oracle.so")
 
-GBA, GSA, SPS, SIMS, GBAD = 0, 1, 2, 3, 4
-FAMILY = {"GBA": GBA, "GSA": GSA, "SPS": SPS, "SIMS": SIMS, "GBAD": GBAD}
+GBA, GSA, SPS, SIMS, GBAD, GSAS = 0, 1, 2, 3, 4, 5
+FAMILY = {"GBA": GBA, "GSA": GSA, "SPS": SPS, "SIMS": SIMS, "GBAD": GBAD, "GSAS": GSAS}
 
 
 def build(force: bool = False) -> str:

@@ -32,6 +32,9 @@
 //   * the dynamic refill of the batching schedule (the paper gives its rule in words; the reading is stated at
 //     `dynamic_refill`; pinned by what the paper promises - no job starts later than in the batching schedule,
 //     every round fits - by a hand-worked instance and by the brute-force optimum as a lower bound),
+//   * speculative runs on top of the slicing schedule (in words in the paper; reading at `speculative_runs`;
+//     pinned by what the paper promises - the slicing schedule is kept, so no job completes later than in it,
+//     and every round fits - by a hand-worked instance and by the brute-force optimum as a lower bound),
 //   * the two variants inside the geometric classes (simultaneous batches as the subroutine of a phase -
 //     pinned by 21632 and Example 1's 225, which the batching algorithm must reproduce when one class holds
 //     every job; per-phase prompt length - pinned by the reduction to one prompt length).
@@ -172,7 +175,7 @@ std::vector<i64> ladder(i64 X, int a, int b, i64 beta0) {
   return tau;
 }
 
-enum { FAM_GBA = 0, FAM_GSA = 1, FAM_SPS = 2, FAM_SIMS = 3, FAM_GBAD = 4 };
+enum { FAM_GBA = 0, FAM_GSA = 1, FAM_SPS = 2, FAM_SIMS = 3, FAM_GBAD = 4, FAM_GSAS = 5 };
 
 struct Run { i64 job, phase, start, len, s; };
 
@@ -252,6 +255,91 @@ void dynamic_refill(Schedule& S, i64 M) {
   }
 }
 
+// Speculative runs on top of a slicing schedule (Numerical Experiments, "Speculative Runs (GSA-Spec)": memory
+// left free by the pipeline is used to run unfinished jobs ahead of their turn; such runs are killed when the
+// pipeline needs the memory, so that the slicing schedule itself is kept; they are started and killed first
+// come first served).  The paper gives this in words; the reading taken here, round by round:
+//   the base runs of the slicing schedule keep their start rounds and lengths; a base run of a job that has
+//   already completed is dropped (it holds nothing);
+//   round t: (1) a speculative run that has received all o rounds completes its job (completion = t);
+//   (2) the base runs that start at t begin - a job that is running speculatively at that moment loses that run
+//   (killed, progress lost); a base run as long as the job's response completes the job at its end, nothing
+//   interrupts base runs; (3) while base and speculative runs together exceed M in round t, the speculative run
+//   started last is killed; (4) jobs that are not done and not running are taken in index order (first come
+//   first served): the first one starts a speculative run at t if its first round fits (s + 1 more tokens in
+//   round t; the scheduler knows no response length), then the next one, until one does not fit.
+// A speculative run holds s + u + 1 tokens in its round u like any other run (Eq. Memory-Feasibility).
+// The schedule's runs are replaced by the executed ones (base runs not dropped, speculative runs with the
+// rounds they received), in order of start round; job results are those of the run that completed the job.
+void speculative_runs(Schedule& S, const int32_t* s, const int32_t* o, i64 M) {
+  const i64 n = S.n;
+  const std::vector<Run> base = S.runs;                 // (phase, rank) order: start rounds nondecreasing
+  std::vector<Run> exec;
+  std::vector<char> done(static_cast<size_t>(n), 0);
+  std::vector<i64> base_end(static_cast<size_t>(n), 0), spec_start(static_cast<size_t>(n), -1);
+  std::vector<i64> spec;                                // jobs running speculatively, in order of their starts
+  struct Active { i64 job, start, len; };
+  std::vector<Active> act;                              // base runs in progress
+  size_t next = 0;
+  i64 left = n;
+  for (i64 t = 0; left > 0 || next < base.size(); ++t) {
+    // (1) speculative completions
+    for (size_t q = 0; q < spec.size();) {
+      const i64 i = spec[q];
+      if (spec_start[i] + o[i] == t) {
+        exec.push_back(Run{i, -1, spec_start[i], o[i], s[i]});
+        S.job_start[i] = spec_start[i]; S.job_completion[i] = t;
+        done[i] = 1; --left; spec_start[i] = -1;
+        spec.erase(spec.begin() + static_cast<std::ptrdiff_t>(q));
+      } else {
+        ++q;
+      }
+    }
+    // base runs that have ended
+    for (size_t q = 0; q < act.size();) { if (act[q].start + act[q].len <= t) act.erase(act.begin() + static_cast<std::ptrdiff_t>(q)); else ++q; }
+    // (2) base runs that start now
+    while (next < base.size() && base[next].start == t) {
+      const Run& r = base[next++];
+      const i64 i = r.job;
+      if (done[i]) continue;                            // dropped
+      if (spec_start[i] >= 0) {                         // its speculative run is killed
+        exec.push_back(Run{i, -1, spec_start[i], t - spec_start[i], s[i]});
+        spec.erase(std::find(spec.begin(), spec.end(), i));
+        spec_start[i] = -1;
+      }
+      exec.push_back(r);
+      act.push_back(Active{i, t, r.len});
+      base_end[i] = t + r.len;
+      if (r.len == o[i]) { done[i] = 1; --left; S.job_start[i] = t; S.job_completion[i] = t + r.len; }
+    }
+    // memory of round t
+    auto memory = [&]() {
+      i64 m = 0;
+      for (const Active& a : act) m += s[a.job] + (t - a.start) + 1;
+      for (i64 i : spec) m += s[i] + (t - spec_start[i]) + 1;
+      return m;
+    };
+    // (3) the pipeline comes first
+    while (!spec.empty() && memory() > M) {
+      const i64 i = spec.back();
+      exec.push_back(Run{i, -1, spec_start[i], t - spec_start[i], s[i]});
+      spec_start[i] = -1;
+      spec.pop_back();
+    }
+    // (4) first come first served
+    for (i64 i = 0; i < n; ++i) {
+      if (done[i] || spec_start[i] >= 0 || base_end[i] > t) continue;
+      if (memory() + s[i] + 1 > M) break;
+      spec_start[i] = t;
+      spec.push_back(i);
+    }
+  }
+  // runs that received no round (killed in the round they started) are not runs
+  exec.erase(std::remove_if(exec.begin(), exec.end(), [](const Run& r) { return r.len <= 0; }), exec.end());
+  std::stable_sort(exec.begin(), exec.end(), [](const Run& x, const Run& y) { return x.start < y.start; });
+  S.runs = exec;
+}
+
 Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int32_t* o_est,
                 const i64* arrival, i64 M, int a, int b, i64 beta0, i64 s_bar_in, i64 tau_in,
                 i64 k_in, i64 window, int subroutine = 0, int per_class = 0) {
@@ -259,7 +347,12 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
   S->n = n;
   S->job_start.assign(n, -1);
   S->job_completion.assign(n, -1);
-  bool refill = false;
+  bool refill = false, speculate = false;
+  if (family == FAM_GSAS) {
+    if (o_est || window != 0 || subroutine != 0) { S->status = 3; return S; }   // speculation is defined on the plain slicing schedule
+    family = FAM_GSA;
+    speculate = true;
+  }
   if (family == FAM_GBAD) {
     if (o_est || window != 0 || subroutine != 0) { S->status = 3; return S; }   // the refill is defined on the plain batching schedule
     family = FAM_GBA;
@@ -355,6 +448,7 @@ Schedule* build(int family, i64 n, const int32_t* s, const int32_t* o, const int
   }
 
   if (refill && S->status == 0) dynamic_refill(*S, M);
+  if (speculate && S->status == 0) speculative_runs(*S, s, o, M);
   for (const Run& r : S->runs) {
     S->horizon = std::max(S->horizon, r.start + r.len);
     S->job_steps += r.len;

@@ -527,3 +527,66 @@ def test_dynamic_refill_keeps_the_paper_promises():
     D = oracle.build_schedule("GBAD", [0] * 5, [8] * 5, 8)
     assert list(D.job_start) == [0, 8, 16, 24, 32]
     assert oracle.build_schedule("GBAD", [1], [1], 10, window=5).status == 3
+
+
+# ---- speculative runs on top of the slicing schedule ----------------------------------------------
+
+def test_speculative_runs_hand_worked_instance(golden_dir):
+    """M = 6, s = 0, o = 4, 4, 2 (alpha = 2: slices 1, 3, 6 with k* = 3, 3, 1).  By hand from the reading:
+    round 0 the three unit runs; round 1 job 0 starts its slice of 3 and jobs 1, 2 (free, 1 + 1 + 1 <= 6) start
+    speculative runs; round 2 job 1's slice starts, so its speculative run is killed after one round; round 3
+    job 2's speculative run has its 2 rounds: done at 3 (5 in the slicing schedule), its slice of round 3 is
+    dropped; rounds 4 and 5 jobs 0 and 1 come free and speculate; round 6 job 0's slice of 6 starts and kills
+    its speculative run (2 rounds); round 8 the slice holds 3 and job 1's speculative run 4 > 6: killed after 3
+    rounds, and, being free and first in line, restarted at once (3 + 1 <= 6); it completes at 12 (16 in the
+    slicing schedule), job 0 at 10 as planned.  Flow 25 against 31."""
+    rows = [ln.split() for ln in open(os.path.join(golden_dir, "speculative_runs_hand_example.txt")) if ln.strip() and not ln.startswith("#")]
+    want = {r[0]: [int(x) for x in r[1:]] for r in rows if r[0] != "run"}
+    runs = [tuple(int(x) for x in r[1:]) for r in rows if r[0] == "run"]
+    n = len(want["o"])
+    G = oracle.build_schedule("GSA", [0] * n, want["o"], 6)
+    assert list(G.job_completion) == want["gsa_completion"]
+    S = oracle.build_schedule("GSAS", [0] * n, want["o"], 6)
+    assert S.status == 0 and S.n_unfinished == 0
+    assert list(S.job_start) == want["start"] and list(S.job_completion) == want["completion"] and S.flow == want["flow"][0]
+    assert list(zip(S.run_job.tolist(), S.run_start.tolist(), S.run_len.tolist())) == runs
+    assert list(_dense(S).profile) == want["memory"]
+    assert S.job_steps == sum(r[2] for r in runs)
+
+
+def test_speculative_runs_keep_the_paper_promises():
+    """The slicing schedule is kept: every pipeline run of a job that has not completed by then is executed at
+    its round and length, so no job completes later than in the slicing schedule; every round fits; the flow
+    time is at least the optimum; an instance whose pipeline leaves no room for a further first round is
+    unchanged."""
+    rng = np.random.default_rng(97)
+    improved = 0
+    for alpha in [(2, 1), (3, 2)]:
+        for it in range(120):
+            s, o, M = _random_instance(rng, hetero=it % 3 == 0)
+            G = oracle.build_schedule("GSA", s, o, M, alpha=alpha)
+            S = oracle.build_schedule("GSAS", s, o, M, alpha=alpha)
+            assert S.status == 0 and S.n_unfinished == 0
+            assert np.all(S.job_completion <= G.job_completion) and S.flow <= G.flow
+            improved += S.flow < G.flow
+            assert _dense(S).peak <= M and np.all(np.diff(S.run_start) >= 0)
+            ex = set(zip(S.run_job.tolist(), S.run_start.tolist(), S.run_len.tolist()))
+            for j, t0, ln in zip(G.run_job.tolist(), G.run_start.tolist(), G.run_len.tolist()):
+                if S.job_completion[j] > t0:            # not done when the pipeline reaches it (a run that completes
+                    assert (j, t0, ln) in ex            # its job at t0 + len has completion > t0 as well)
+            # the run that completes a job has its full length; every run's length is at most the job's
+            done_runs = {(j, c - ln) for j, c, ln in zip(range(len(o)), S.job_completion.tolist(), np.asarray(o).tolist())}
+            assert all((j, t0, int(o[j])) in ex for j, t0 in done_runs)
+            assert np.all(S.run_len <= np.asarray(o)[S.run_job]) and S.job_steps >= int(np.sum(o))
+    assert improved > 60
+    for it in range(60):
+        n, s = int(rng.integers(1, 8)), int(rng.integers(0, 6))
+        o = rng.integers(1, 7, n)
+        M = int(s + o.max() + rng.integers(0, 14))
+        assert oracle.opt_bruteforce(s, o, M) <= oracle.build_schedule("GSAS", [s] * n, o, M).flow
+    # one job at a time fills the memory: nothing can be added
+    A, B = oracle.build_schedule("GSA", [7] * 3, [1] * 3, 8), oracle.build_schedule("GSAS", [7] * 3, [1] * 3, 8)
+    assert _same(A, B)
+    # a single job is its own pipeline
+    assert _same(oracle.build_schedule("GSA", [3], [9], 40), oracle.build_schedule("GSAS", [3], [9], 40))
+    assert oracle.build_schedule("GSAS", [1], [1], 10, window=5).status == 3
