@@ -467,11 +467,27 @@ def run_fused_workload(args, rank, world, dev, local, dist, binding, Scheduler):
                                   None if inst.o_est is None else inst.o_est.cpu().pin_memory(),
                                   None if inst.arrival is None else inst.arrival.cpu().pin_memory())
         hev = {k: torch.zeros_like(v, device="cpu").pin_memory() for k, v in Scheduler.scalars(P, "cpu").items()}
-        ctx.evaluate_built_host(hin, settings, hev, window=window, max_jobs=n)
+        # The refill and the speculative runs work in the per-job results and the profile on the device, which the
+        # host entry point does not allocate: their end-to-end step copies the pinned inputs to the device, calls
+        # the device entry point and copies the scalars back.
+        on_device = bool(np.isin(settings["family"], [binding.FAMILY[f] for f in ("GBAD", "GSAS") if f in binding.FAMILY]).any())
+
+        def e2e_step():
+            if not on_device:
+                ctx.evaluate_built_host(hin, settings, hev, window=window, max_jobs=n)
+                return
+            din = workloads.Instances(*[None if x is None else x.to(dev, non_blocking=True)
+                                        for x in (hin.job_off, hin.s, hin.o, hin.o_est, hin.arrival)])
+            ctx.evaluate_built(din, settings, out, ev, window=window, max_jobs=n)
+            for k2, v2 in hev.items():
+                v2.copy_(ev[k2], non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_step()
         barrier()
         t0 = time.perf_counter()
         for _ in range(args.steps):
-            ctx.evaluate_built_host(hin, settings, hev, window=window, max_jobs=n)
+            e2e_step()
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
         assert int(hev["job_steps"].sum()) == job_steps

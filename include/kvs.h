@@ -53,7 +53,17 @@ enum kvs_family { KVS_GBA = 0, KVS_GSA = 1, KVS_SPS = 2, KVS_SIMS = 3,
                    * profile with the batching schedule's horizon as capacity: they are its working storage) and by
                    * kvs_build_schedule (which reports the batching schedule: its horizon sizes the profile); offline
                    * instances without estimates only. */
-                  KVS_GBAD = 4 };
+                  KVS_GBAD = 4,
+                  /* GSA with speculative runs (Numerical Experiments, "Speculative Runs (GSA-Spec)"): the slicing
+                   * schedule is formed first and kept; round by round, memory it leaves free starts further runs of
+                   * jobs that are neither done nor running, lowest index first, as long as the first round of the
+                   * next one fits; when the schedule's own runs need the memory the speculative run started last is
+                   * killed; a job completed by a speculative run drops out of the schedule's later phases.  No job
+                   * completes later than in the slicing schedule.  Accepted like KVS_GBAD (job_start, job_completion
+                   * and a profile with the slicing schedule's horizon as capacity are the working storage;
+                   * kvs_build_schedule reports the slicing schedule); offline instances without estimates, staggered
+                   * subroutine, one prompt length for the parallelism. */
+                  KVS_GSAS = 5 };
 
 /* Bits of the per-evaluation status word. */
 enum kvs_eval_status {

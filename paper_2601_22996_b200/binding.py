@@ -17,8 +17,8 @@ import torch
 from . import build as _build
 from .workloads import Instances
 
-GBA, GSA, SPS, SIMS, GBAD = 0, 1, 2, 3, 4
-FAMILY = {"GBA": GBA, "GSA": GSA, "SPS": SPS, "SIMS": SIMS, "GBAD": GBAD}
+GBA, GSA, SPS, SIMS, GBAD, GSAS = 0, 1, 2, 3, 4, 5
+FAMILY = {"GBA": GBA, "GSA": GSA, "SPS": SPS, "SIMS": SIMS, "GBAD": GBAD, "GSAS": GSAS}
 EVAL_OK, EVAL_INFEASIBLE, EVAL_RANGE, EVAL_CAPACITY, EVAL_BAD_INPUT = 0, 1, 2, 4, 8
 
 SETTING_DTYPE = np.dtype([("instance", "<i8"), ("family", "<i4"), ("alpha_num", "<i4"), ("alpha_den", "<i4"),
@@ -172,7 +172,7 @@ def settings_grid(instances, families, Ms, alpha=(2, 1), subroutine=0, per_class
     out["M"] = Ms[None, :, None] if Ms.ndim == 1 else Ms[:, :, None]
     out["alpha_num"], out["alpha_den"] = alpha
     out["s_bar"] = -1
-    geo = (out["family"] <= GSA) | (out["family"] == GBAD)
+    geo = (out["family"] <= GSA) | (out["family"] >= GBAD)
     out["subroutine"] = np.where(geo, subroutine, 0)
     out["per_class_s"] = np.where(geo, per_class_s, 0)
     return out.reshape(-1)

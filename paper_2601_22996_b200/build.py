@@ -10,7 +10,7 @@ _CSRC = os.path.join(_HERE, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libkvs.so")
 DEBUG_LIB_PATH = os.path.join(_HERE, "libkvs_debug.so")   # the same sources with -DKVS_DEBUG (index checks)
-SOURCES = ["kvs_api.cu", "kvs_sort.cu", "kvs_build.cu", "kvs_fused.cu", "kvs_refill.cu", "kvs_bounds.cu", "kvs_generic.cu", "kvs_sweep.cu"]
+SOURCES = ["kvs_api.cu", "kvs_sort.cu", "kvs_build.cu", "kvs_fused.cu", "kvs_refill.cu", "kvs_spec.cu", "kvs_bounds.cu", "kvs_generic.cu", "kvs_sweep.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", _INCLUDE, "-I", _CSRC]
 

@@ -160,7 +160,9 @@ int check_settings(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* s
   for (int64_t e = 0; e < P; ++e) {
     const kvs_setting& s = st[e];
     if (s.instance < 0 || s.instance >= inst->n_instances) return fail(ctx, KVS_E_ARG, "settings: instance out of range");
-    if (s.family < KVS_GBA || s.family > KVS_GBAD) return fail(ctx, KVS_E_ARG, "settings: unknown family");
+    if (s.family < KVS_GBA || s.family > KVS_GSAS) return fail(ctx, KVS_E_ARG, "settings: unknown family");
+    if (s.family == KVS_GSAS && (inst->o_est || inst->window != 0 || s.subroutine || s.per_class_s))
+      return fail(ctx, KVS_E_ARG, "settings: speculative runs take offline instances without estimates and the plain slicing schedule");
     if (s.family == KVS_GBAD && (inst->o_est || inst->window != 0 || s.subroutine))
       return fail(ctx, KVS_E_ARG, "settings: the dynamic refill takes offline instances without estimates and the staggered subroutine");
     if (s.M < 1 || s.M >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: M outside [1, 2^31)");
@@ -169,9 +171,9 @@ int check_settings(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* s
       return fail(ctx, KVS_E_RANGE, "settings: tau or k outside [0, 2^31)");
     if (s.subroutine < 0 || s.subroutine > 1 || s.per_class_s < 0 || s.per_class_s > 1)
       return fail(ctx, KVS_E_ARG, "settings: subroutine and per_class_s are 0 or 1");
-    if ((s.subroutine || s.per_class_s) && s.family != KVS_GBA && s.family != KVS_GSA && s.family != KVS_GBAD)
+    if ((s.subroutine || s.per_class_s) && s.family != KVS_GBA && s.family != KVS_GSA && s.family != KVS_GBAD && s.family != KVS_GSAS)
       return fail(ctx, KVS_E_ARG, "settings: subroutine and per_class_s apply to the geometric families only");
-    if (s.family == KVS_GBA || s.family == KVS_GSA || s.family == KVS_GBAD) {
+    if (s.family == KVS_GBA || s.family == KVS_GSA || s.family == KVS_GBAD || s.family == KVS_GSAS) {
       if (s.alpha_den < 1 || s.alpha_num <= s.alpha_den) return fail(ctx, KVS_E_ARG, "settings: alpha must be > 1");
       if (s.beta0 < 0 || s.beta0 >= KVS_TIME_LIMIT) return fail(ctx, KVS_E_RANGE, "settings: beta0 outside [0, 2^31)");
       if (!(s.alpha_num == 2 && s.alpha_den == 1) && !ladder_fits(s.M, s.alpha_num, s.alpha_den))
@@ -205,15 +207,21 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
   if (!do_profile) v.profile = nullptr;
   if (P == 0) return KVS_OK;
   // Dynamic refill: the fused kernels form the batching schedule; a last kernel refills it in place.
-  std::vector<int64_t> refill;
-  for (int64_t e = 0; e < P; ++e)
+  // Speculative runs: the same on top of the slicing schedule.
+  std::vector<int64_t> refill, spec;
+  for (int64_t e = 0; e < P; ++e) {
     if (settings[e].family == KVS_GBAD) refill.push_back(e);
-  if (!refill.empty()) {
-    if (rg) return fail(ctx, KVS_E_ARG, "the host entry point does not take the dynamic refill (it needs per-job results and a profile on the device)");
+    if (settings[e].family == KVS_GSAS) spec.push_back(e);
+  }
+  if (!refill.empty() || !spec.empty()) {
+    if (rg) return fail(ctx, KVS_E_ARG, "the host entry point takes neither the dynamic refill nor speculative runs (they need per-job results and a profile on the device)");
     if (do_profile && (!o.job_start || !o.job_completion || !v.profile || o.job_start64 || o.job_completion64 || run_out))
-      return fail(ctx, KVS_E_ARG, "the dynamic refill needs job_start, job_completion and a profile (32-bit, no run list): they are its working storage");
+      return fail(ctx, KVS_E_ARG, "the dynamic refill and speculative runs need job_start, job_completion and a profile (32-bit, no run list): they are their working storage");
+    if (do_profile && (!v.horizon || !v.status))
+      return fail(ctx, KVS_E_ARG, "the dynamic refill and speculative runs need the horizon and status outputs");
     ctx->settings_tmp.assign(settings, settings + P);
     for (int64_t e : refill) ctx->settings_tmp[static_cast<size_t>(e)].family = KVS_GBA;
+    for (int64_t e : spec) ctx->settings_tmp[static_cast<size_t>(e)].family = KVS_GSA;
     settings = ctx->settings_tmp.data();
   }
 
@@ -385,9 +393,31 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     rp.job_out_off = o.job_out_off; rp.job_start = o.job_start; rp.job_completion = o.job_completion;
     rp.profile_off = v.profile_off; rp.profile = v.profile;
     rp.peak = v.peak; rp.flow = v.flow; rp.horizon = v.horizon; rp.feasible = v.feasible; rp.status = v.status;
-    if (!v.horizon || !v.status) return fail(ctx, KVS_E_ARG, "the dynamic refill needs the horizon and status outputs");
     ce = kvs_launch_refill(rp, ctx->stream);
     if (ce != cudaSuccess) return fail_cuda(ctx, ce, "refill launch");
+  }
+  if (do_profile && !spec.empty()) {
+    // the list shares the refill list's region (together at most P entries); the working storage is the fused
+    // kernels' per-CTA scratch, free once they have run
+    unsigned char* const list_dev = ws + L.refill_list + refill.size() * 8;
+    ce = cudaMemcpyAsync(list_dev, spec.data(), spec.size() * 8, cudaMemcpyHostToDevice, ctx->stream);
+    if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of the list of speculative evaluations");
+    SpecParams q{};
+    q.job_off = inst->job_off; q.s = inst->s; q.o = inst->o;
+    q.stats = reinterpret_cast<const InstStats*>(ws + L.stats);
+    q.settings = reinterpret_cast<const kvs_setting*>(settings_dev);
+    q.eval_list = reinterpret_cast<const i64*>(list_dev); q.n_list = static_cast<i64>(spec.size());
+    q.job_out_off = o.job_out_off; q.job_start = o.job_start; q.job_completion = o.job_completion;
+    q.profile_off = v.profile_off; q.profile = v.profile;
+    q.peak = v.peak; q.flow = v.flow; q.horizon = v.horizon; q.job_steps = v.job_steps; q.n_runs = o.n_runs;
+    q.n_unfinished = v.n_unfinished; q.feasible = v.feasible; q.status = v.status;
+    q.scratch = ws + L.lists; q.max_jobs = max_n;
+    const i64 room = static_cast<i64>(L.counter - L.lists) / kvs_spec_warp_bytes(max_n);
+    const i64 want = static_cast<i64>(ctx->sm_count) * 32;
+    q.n_warps = std::min<i64>(std::min<i64>(room, want), q.n_list);
+    q.counter = counters + 24;
+    ce = kvs_launch_spec(q, ctx->stream);
+    if (ce != cudaSuccess) return fail_cuda(ctx, ce, "launch of the speculative runs");
   }
   if (ctx->timing && !rg) { cudaEventRecord(ctx->ev[2], ctx->stream); ctx->timed = true; ctx->split_timed = fast; }
   return KVS_OK;

@@ -124,6 +124,28 @@ struct RefillParams {
   const int32_t* status;
 };
 
+// Speculative runs on top of the slicing schedules of the listed evaluations, in place (see kvs_spec.cu).
+struct SpecParams {
+  const i64* job_off;
+  const int32_t* s;            // prompt and response lengths in index order
+  const int32_t* o;
+  const InstStats* stats;
+  const kvs_setting* settings;
+  const i64* eval_list;        // evaluations to work on
+  i64 n_list;
+  const i64* job_out_off;
+  int32_t* job_start;          // in: of the slicing schedule; out: of the run that completed the job
+  int32_t* job_completion;
+  const i64* profile_off;
+  int32_t* profile;            // in: memory of the slicing schedule; out: with the speculative runs
+  i64* peak; i64* flow; i64* horizon; i64* job_steps; i64* n_runs; i64* n_unfinished; uint8_t* feasible;
+  const int32_t* status;
+  unsigned char* scratch;      // n_warps blocks of kvs_spec_warp_bytes(max_jobs) bytes
+  i64 max_jobs;
+  i64 n_warps;                 // warps launched; each takes evaluations from the list until it is used up
+  ull* counter;
+};
+
 struct SweepParams {
   const int32_t* sorted_s;  // the instance in key order
   const int32_t* sorted_o;
@@ -147,6 +169,8 @@ int kvs_fused_ctas_per_sm(int light);
 cudaError_t kvs_fused_check_word(unsigned long long* word, int* compiled, int reset);
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_refill(const RefillParams& p, cudaStream_t stream);
+i64 kvs_spec_warp_bytes(i64 max_jobs);
+cudaError_t kvs_launch_spec(const SpecParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_bounds(const i64* job_off, const int32_t* o, const InstStats* stats, const kvs_setting* settings,
                               i64 P, const kvs_bounds_out& out, int grid, cudaStream_t stream);
 cudaError_t kvs_launch_prefix(const int32_t* sorted_s, const int32_t* sorted_o, i64 n, i64* prefix_s,

@@ -1,0 +1,317 @@
+// Speculative runs on top of slicing schedules (Numerical Experiments, "Speculative Runs (GSA-Spec)"): memory
+// that the pipeline leaves free runs unfinished jobs ahead of their turn; such runs are killed when the
+// pipeline needs the memory, so the slicing schedule itself is kept; they start and are killed first come
+// first served.
+//
+// The rule is a round-by-round simulation in which every decision depends on the rounds before it, so one
+// warp simulates one evaluation and many evaluations run side by side.  The warp starts from what the fused
+// kernels left - the per-round memory of the slicing schedule (the plan) in the caller's profile buffer -
+// and forms the pipeline's runs again from the phase table: the participants of phase p are the jobs of class
+// p or later in index order, rank r starts at base_p + floor(r tau_p / k_p) and holds its slot for tau_p rounds
+// (Procedure StaggeredPipelineSchedule).  Round t:
+//   (1) a speculative run that has received all its rounds completes its job;
+//   (2) the pipeline's runs that start at t begin: a job that has completed is dropped from the plan (its ramp
+//       is taken out of the profile), a job that is running speculatively loses that run;
+//   (3) while pipeline and speculative runs together exceed M, the speculative run started last is killed;
+//   (4) the jobs that are not done and not running are taken in index order: the lowest one starts a
+//       speculative run if its first round fits (s + 1 tokens), then the next, until one does not fit;
+//   (5) the round's memory, pipeline + speculative, is written over the plan's entry.
+// The speculative runs hold A + t * count tokens in round t (a run started at t0 holds s + 1 - t0 + t).
+// Per phase the participants are kept as a list in index order, so that rank r is entry r.  Two cursors walk
+// it: one over the run starts, one over the slot ends start + tau (nondecreasing in the rank), which is when a
+// killed job becomes free to speculate.  `fpos` is a position such that no entry before it is free at the
+// moment; the events that free a job (a slot end, a kill for memory) lower it.
+#include "kvs_ladder.cuh"
+
+namespace {
+
+constexpr int ST = 128;                 // threads per CTA: four warps, one evaluation each at a time
+constexpr int SWARPS = ST / 32;
+constexpr int MAXP = KVS_MAX_PHASES;
+constexpr int NEVER = 0x7fffffff;
+
+struct SpecShared {
+  u128 pw_a[MAXP + 1];
+  u128 pw_b[MAXP + 1];
+  u32 tau[MAXP], k[MAXP], np[MAXP], hist[MAXP];
+  i64 pbase[MAXP + 1];
+  int n_phases;
+};
+
+// floor(r * tau / k) for r, tau, k below 2^31
+__device__ __forceinline__ i64 slot_of(int r, u32 tau, u32 k) {
+  const u64 x = static_cast<u64>(static_cast<u32>(r)) * tau;
+  return (x >> 32) == 0 ? static_cast<i64>(static_cast<u32>(x) / k) : static_cast<i64>(x / k);
+}
+
+__device__ __forceinline__ int warp_min_int(int v) { return -warp_max(-v); }
+
+// Bytes of one warp's working storage for instances of at most n jobs: five int arrays (end of the latest
+// pipeline run, start of the speculative run or -1, stack of speculative runs as job and start, participant
+// list) and two byte arrays (class, done flag).
+__host__ __device__ inline i64 spec_stride(i64 n) { return (22 * n + 255) & ~static_cast<i64>(255); }
+
+__global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
+  __shared__ SpecShared shs[SWARPS];
+  const int lane = lane_id(), warp = threadIdx.x >> 5;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  SpecShared& sh = shs[warp];
+  const i64 wslot = static_cast<i64>(blockIdx.x) * SWARPS + warp;
+  if (wslot >= p.n_warps) return;
+  const i64 cap = p.max_jobs;
+  unsigned char* const mine = p.scratch + wslot * spec_stride(cap);
+  int* const be = reinterpret_cast<int*>(mine);
+  int* const sst = be + cap;
+  int* const stk_job = sst + cap;
+  int* const stk_start = stk_job + cap;
+  int* const list = stk_start + cap;
+  unsigned char* const cls = reinterpret_cast<unsigned char*>(list + cap);
+  unsigned char* const done = cls + cap;
+
+  for (;;) {
+    ull slot = 0;
+    if (lane == 0) slot = atomicAdd(p.counter, 1ull);
+    slot = __shfl_sync(0xffffffffu, slot, 0);
+    if (slot >= static_cast<ull>(p.n_list)) return;
+    const i64 e = p.eval_list[slot];
+    if (p.status[e] != 0) continue;                     // the slicing schedule was not formed or not stored in full
+    const kvs_setting st = p.settings[e];
+    const i64 lo = p.job_off[st.instance];
+    const int n = static_cast<int>(p.job_off[st.instance + 1] - lo);
+    const InstStats stats = p.stats[st.instance];
+    const i64 M = st.M;
+    const i64 s_bar = st.s_bar >= 0 ? st.s_bar : stats.s_max;
+    const i64 X = M - s_bar;
+    const int32_t* const S = p.s + lo;
+    const int32_t* const O = p.o + lo;
+    int32_t* const prof = p.profile + p.profile_off[e];
+    int32_t* const js = p.job_start + p.job_out_off[e];
+    int32_t* const jc = p.job_completion + p.job_out_off[e];
+    const int H = static_cast<int>(p.horizon[e]);       // of the slicing schedule; within the profile's capacity (status 0)
+    if (n == 0) continue;
+
+    // ---- phase table: ladder, classes, participants, first round of every phase ----
+    ladder32(sh, X, st.alpha_num, st.alpha_den, st.beta0, static_cast<u32>(s_bar), static_cast<u32>(M));
+    const int L = sh.n_phases;
+    for (int q = lane; q < L; q += 32) sh.hist[q] = 0;
+    __syncwarp();
+    const bool pow2 = st.alpha_num == 2 && st.alpha_den == 1 && st.beta0 <= 0;
+    for (int i = lane; i < n; i += 32) {
+      const u32 oi = static_cast<u32>(O[i]);
+      const int c = pow2 ? class_pow2(static_cast<u32>(X), oi) : class_of(sh.tau, L, oi);
+      cls[i] = static_cast<unsigned char>(c);
+      done[i] = 0; be[i] = 0; sst[i] = -1; list[i] = i;
+      atomicAdd(&sh.hist[c], 1u);
+    }
+    __syncwarp();
+    if (lane == 0) {
+      u32 later = static_cast<u32>(n);
+      i64 b = 0;
+      for (int q = 0; q < L; ++q) {
+        sh.np[q] = later;                               // jobs of class q or later take part in phase q
+        sh.pbase[q] = b;
+        if (later > 0) b += slot_of(static_cast<int>(later) - 1, sh.tau[q], sh.k[q]) + sh.tau[q];
+        later -= sh.hist[q];
+      }
+      sh.pbase[L] = b;
+    }
+    __syncwarp();
+
+    // ---- the simulation ----
+    int ph = 0, np = n;                                 // phase that holds round t; its participants
+    u32 tau_c = sh.tau[0], k_c = sh.k[0];
+    i64 base_c = 0;
+    int rs = 0, re = 0;                                 // ranks of the next run start and of the next slot end
+    i64 ns = 0, ne = tau_c;                             // their rounds
+    i64 A = 0;                                          // speculative runs hold A + t * cnt tokens in round t
+    int cnt = 0, top = 0;                               // running speculative runs; entries on the stack (some stale)
+    int next_comp = NEVER;                              // no speculative run completes before this round
+    int fpos = 0;
+    int left = n;
+    i64 flow = 0, steps = 0, runs = 0, peak = 0;
+    int hmax = 0;
+    int Bw = 0;                                         // lane l holds the plan's memory of round (t & ~31) + l
+    for (int t = 0; t <= H; ++t) {
+      // (1) speculative completions
+      if (t == next_comp) {
+        int nc = NEVER;
+        for (int q0 = 0; q0 < top; q0 += 32) {
+          const int q = q0 + lane;
+          bool fin = false;
+          int j = 0, s0 = 0;
+          if (q < top) {
+            j = stk_job[q]; s0 = stk_start[q];
+            if (sst[j] == s0) {                         // a live entry
+              const int f = s0 + O[j];
+              if (f == t) fin = true; else nc = min(nc, f);
+            }
+          }
+          const unsigned fm = __ballot_sync(0xffffffffu, fin);
+          if (fm) {
+            if (fin) { done[j] = 1; sst[j] = -1; js[j] = s0; jc[j] = t; }
+            const i64 dA = warp_sum(fin ? static_cast<i64>(S[j]) + 1 - s0 : static_cast<i64>(0));
+            const i64 dS = warp_sum(fin ? static_cast<i64>(O[j]) : static_cast<i64>(0));
+            const int kf = __popc(fm);
+            A -= dA; steps += dS; flow += static_cast<i64>(kf) * t;
+            cnt -= kf; left -= kf; runs += kf;
+            hmax = max(hmax, t);
+          }
+        }
+        next_comp = warp_min_int(nc);
+        __syncwarp();
+      }
+      // slots that have ended: a job killed at the end of its slot is free again
+      while (ne <= t) {
+        const int j = list[re];
+        if (!done[j] && sst[j] < 0) fpos = min(fpos, re);
+        ++re;
+        ne = re < np ? base_c + slot_of(re, tau_c, k_c) + tau_c : static_cast<i64>(NEVER) * 2;
+      }
+      // the next phase begins: its participants are the jobs of a later class, in index order
+      if (rs >= np && ph + 1 < L && sh.np[ph + 1] > 0 && t == sh.pbase[ph + 1]) {
+        ++ph;
+        int w = 0;
+        for (int q0 = 0; q0 < np; q0 += 32) {
+          const int q = q0 + lane;
+          bool keep = false;
+          int j = 0;
+          if (q < np) { j = list[q]; keep = cls[j] >= ph; }
+          const unsigned m = __ballot_sync(0xffffffffu, keep);
+          __syncwarp();
+          if (keep) list[w + __popc(m & lt_mask)] = j;
+          w += __popc(m);
+          __syncwarp();
+        }
+        np = w;
+        tau_c = sh.tau[ph]; k_c = sh.k[ph]; base_c = sh.pbase[ph];
+        rs = 0; re = 0; ns = base_c; ne = base_c + tau_c;
+        fpos = 0;
+      }
+      // (2) pipeline runs that start now
+      bool dropped = false;
+      while (ns <= t) {
+        const int j = list[rs];
+        const int oj = O[j], sj = S[j];
+        const int len = oj < static_cast<int>(tau_c) ? oj : static_cast<int>(tau_c);
+        if (done[j]) {
+          for (int u = lane; u < len; u += 32) prof[t + u] -= sj + u + 1;     // dropped from the plan
+          dropped = true;
+        } else {
+          const int s0 = sst[j];
+          __syncwarp();
+          if (s0 >= 0) {                                // its speculative run is killed; the stack entry goes stale
+            A -= static_cast<i64>(sj) + 1 - s0;
+            --cnt;
+            steps += t - s0;
+            runs += t > s0 ? 1 : 0;
+          }
+          steps += len; ++runs;
+          if (lane == 0) {
+            sst[j] = -1;
+            be[j] = t + len;
+            if (len == oj) { done[j] = 1; js[j] = t; jc[j] = t + len; }
+          }
+          if (len == oj) { --left; flow += t + len; hmax = max(hmax, t + len); }
+          __syncwarp();
+        }
+        ++rs;
+        ns = rs < np ? base_c + slot_of(rs, tau_c, k_c) : static_cast<i64>(NEVER) * 2;
+      }
+      if (t == H) break;                                // nothing runs in round H; only completions were due
+      if ((t & 31) == 0 || dropped) {
+        __syncwarp();
+        const int u = (t & ~31) + lane;
+        Bw = u < H ? prof[u] : 0;
+      }
+      const i64 B = __shfl_sync(0xffffffffu, Bw, t & 31);
+      // (3) the pipeline comes first
+      while (cnt > 0 && B + A + static_cast<i64>(t) * cnt > M) {
+        int j = -1, s0 = 0;
+        while (top > 0) {                               // the live entry nearest to the top
+          --top;
+          const int jj = stk_job[top];
+          s0 = stk_start[top];
+          if (sst[jj] == s0) { j = jj; break; }
+        }
+        if (j < 0) break;
+        __syncwarp();
+        A -= static_cast<i64>(S[j]) + 1 - s0;
+        --cnt;
+        steps += t - s0;
+        runs += t > s0 ? 1 : 0;
+        if (lane == 0) sst[j] = -1;
+        __syncwarp();
+        int a = 0, b = np;                              // its position in the list (ascending job indices)
+        while (a < b) { const int m = (a + b) >> 1; if (list[m] < j) a = m + 1; else b = m; }
+        fpos = min(fpos, a);
+      }
+      // (4) first come first served
+      for (;;) {
+        int c = -1;
+        while (fpos < np) {
+          const int q = fpos + lane;
+          bool fr = false;
+          if (q < np) { const int j = list[q]; fr = !done[j] && sst[j] < 0 && be[j] <= t; }
+          const unsigned hit = __ballot_sync(0xffffffffu, fr);
+          if (hit) { fpos += __ffs(static_cast<int>(hit)) - 1; c = fpos; break; }
+          fpos += 32;
+        }
+        if (c < 0) { fpos = np; break; }
+        const int j = list[c];
+        const int sc = S[j];
+        if (B + A + static_cast<i64>(t) * cnt + sc + 1 > M) break;
+        if (top == static_cast<int>(cap)) {             // stale entries fill the stack: keep the live ones, in order
+          int w = 0;
+          for (int q0 = 0; q0 < top; q0 += 32) {
+            const int q = q0 + lane;
+            bool live = false;
+            int jj = 0, s0 = 0;
+            if (q < top) { jj = stk_job[q]; s0 = stk_start[q]; live = sst[jj] == s0; }
+            const unsigned m = __ballot_sync(0xffffffffu, live);
+            __syncwarp();
+            if (live) { const int d = w + __popc(m & lt_mask); stk_job[d] = jj; stk_start[d] = s0; }
+            w += __popc(m);
+            __syncwarp();
+          }
+          top = w;
+        }
+        __syncwarp();
+        if (lane == 0) { sst[j] = t; stk_job[top] = j; stk_start[top] = t; }
+        __syncwarp();
+        ++top;
+        A += static_cast<i64>(sc) + 1 - t;
+        ++cnt;
+        next_comp = min(next_comp, t + O[j]);
+        ++fpos;
+      }
+      // (5) the round's memory
+      const i64 mem = B + A + static_cast<i64>(t) * cnt;
+      if (lane == 0) prof[t] = static_cast<int32_t>(mem);
+      peak = max_i64(peak, mem);
+      if (cnt == 0) top = 0;                            // only stale entries are left
+    }
+    __syncwarp();
+    if (lane == 0) {
+      if (p.peak) p.peak[e] = peak;
+      if (p.flow) p.flow[e] = flow;
+      if (p.job_steps) p.job_steps[e] = steps;
+      if (p.n_runs) p.n_runs[e] = runs;
+      if (p.n_unfinished) p.n_unfinished[e] = left;
+      p.horizon[e] = hmax;
+      if (p.feasible) p.feasible[e] = peak <= M ? 1 : 0;
+    }
+    __syncwarp();
+  }
+}
+
+}  // namespace
+
+i64 kvs_spec_warp_bytes(i64 max_jobs) { return spec_stride(max_jobs); }
+
+cudaError_t kvs_launch_spec(const SpecParams& p, cudaStream_t stream) {
+  if (p.n_list <= 0 || p.n_warps <= 0) return cudaSuccess;
+  const cudaError_t err = cudaMemsetAsync(p.counter, 0, 8, stream);
+  if (err != cudaSuccess) return err;
+  k_spec<<<static_cast<unsigned>((p.n_warps + SWARPS - 1) / SWARPS), ST, 0, stream>>>(p);
+  return cudaGetLastError();
+}

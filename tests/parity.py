@@ -10,7 +10,7 @@ from paper_2601_22996_b200 import binding
 from paper_2601_22996_b200.api import Scheduler
 from paper_2601_22996_b200.workloads import Instances
 
-FAM_NAME = {0: "GBA", 1: "GSA", 2: "SPS", 3: "SIMS", 4: "GBAD"}
+FAM_NAME = {0: "GBA", 1: "GSA", 2: "SPS", 3: "SIMS", 4: "GBAD", 5: "GSAS"}
 DENSE_LIMIT = 6_000_000   # rounds above which the oracle uses its event evaluator (no dense array)
 
 _scheduler = None
