@@ -3,7 +3,7 @@
 path over one batch of seeded synthetic instances).  Prints ONE JSON line on rank 0.
 
     python bench.py --gpus 1 --steps 5 --warmup 3            # config 5, the workload the target is quoted on
-    python bench.py --workload c1|c2|c3|c4|c5|c2d|bounds     # the other configs: c4 = the (tau, k) sweep, c2d = dynamic refill
+    python bench.py --workload c1|c2|c3|c4|c5|c2d|c2s|bounds # the other configs: c4 = the (tau, k) sweep, c2d = dynamic refill, c2s = speculative runs
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
     python bench.py --impl reference                         # the CPU oracle, as it stands, on a bounded sample
 """
@@ -35,6 +35,7 @@ WORKLOADS = {
     "c4": ("config4", 1, 1_000_000, ["SPS", "SIMS"], "config 4: one instance of 1,000,000 jobs, 64 x 64 (tau, k) grid, SPS and SimS, scalars only"),
     "c5": ("config5", 16_384, 50_000, ["GBA", "GSA", "SPS", "SIMS"], "config 5 (stress): 16,384 instances x 50,000 jobs, mixed distributions, M per instance, four families"),
     "c2d": ("config2", 1024, 10_000, ["GBAD"], "config 2's instances and budgets under GBA with dynamic refill (GBA-D): batching schedule, then the refill kernel"),
+    "c2s": ("config2", 1024, 10_000, ["GSAS"], "config 2's instances and budgets under GSA with speculative runs (GSA-Spec): slicing schedule, then the round-by-round kernel"),
     "bounds": ("config2", 1024, 10_000, ["GBA"], "class-size bounds (kvs_bounds) on config 2's instances and budgets"),
 }
 # The sweep is bound by integer arithmetic on inputs that stay in L2: per candidate round (one per run and
@@ -527,9 +528,10 @@ def run_fused_workload(args, rank, world, dev, local, dist, binding, Scheduler):
     # each for all families); the full variant for what the light one passes on; the general kernel on the
     # left-over list
     n_light_fams = sum(f in ("SPS", "SIMS") for f in fams)
-    n_geo_fams = sum(f in ("GBA", "GSA") for f in fams)
+    n_geo_fams = sum(f in ("GBA", "GSA", "GBAD", "GSAS") for f in fams)
+    n_post = sum(f in fams for f in ("GBAD", "GSAS"))     # k_refill / k_spec after the fused kernels
     if inst.o_est is None:
-        launches_per_step = 1 + n_light_fams + n_geo_fams + int(n_light_fams > 0) + 1
+        launches_per_step = 1 + n_light_fams + n_geo_fams + int(n_light_fams > 0) + 1 + n_post
     else:
         launches_per_step = 1 + int(n_light_fams > 0) + int(n_light_fams + n_geo_fams > 0) + 1
     prof_note = ("every evaluation stores its per-round profile" if walked == P else
@@ -549,7 +551,9 @@ def run_fused_workload(args, rank, world, dev, local, dist, binding, Scheduler):
         "evaluations_per_sec": evals_all / sec_per_step,
         "job_steps_per_sec_split": {"with_stored_profile": steps_prof_all / sec_per_step,
                                     "scalars_only_peak_from_run_ends": (steps_all - steps_prof_all) / sec_per_step},
-        "kernels_ms": {"k_stats_sort": sort_avg, "k_fused_eval<light>": light_avg, "k_fused_eval<full>+k_build_eval": full_avg,
+        "kernels_ms": {"k_stats_sort": sort_avg, "k_fused_eval<light>": light_avg,
+                       ("k_fused_eval<full>+k_build_eval+" + ("k_refill" if "GBAD" in fams else "k_spec") if n_post else
+                        "k_fused_eval<full>+k_build_eval"): full_avg,
                        "builder_evaluator_stage": build_avg},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
                      "traffic": traffic, "peak_kind": peak_kind, "kernel": "k_fused_eval<full>", "algorithmic_bytes": alg_bytes,

@@ -98,7 +98,8 @@ int kvs_set_timing(kvs_ctx* ctx, int32_t enabled);
 int kvs_last_timing(kvs_ctx* ctx, float* sort_ms, float* build_ms);
 /* The same with the builder/evaluator stage split: the variant of the fast kernel for evaluations
  * that walk no rounds (`light_ms`) and everything after it - the full variant and the general
- * kernel (`full_ms`).  A call that took the general kernel alone reports it all as `full_ms`. */
+ * kernel, and the refill / speculative-run kernel of a call with such evaluations (`full_ms`).  A call
+ * that took the general kernel alone reports it all as `full_ms`. */
 int kvs_last_timing_split(kvs_ctx* ctx, float* sort_ms, float* light_ms, float* full_ms);
 
 /* Checked build.  A library compiled with -DKVS_DEBUG tests every computed index of the fast fused kernel

@@ -127,6 +127,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
     int cnt = 0, top = 0;                               // running speculative runs; entries on the stack (some stale)
     int next_comp = NEVER;                              // no speculative run completes before this round
     int fpos = 0;
+    int cj = -1, cs = 0;                                // the free job at fpos and its prompt length, while known (cj = -2: none is free)
     int left = n;
     i64 flow = 0, steps = 0, runs = 0, peak = 0;
     int hmax = 0;
@@ -163,7 +164,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
       // slots that have ended: a job killed at the end of its slot is free again
       while (ne <= t) {
         const int j = list[re];
-        if (!done[j] && sst[j] < 0) fpos = min(fpos, re);
+        if (!done[j] && sst[j] < 0 && re < fpos) { fpos = re; cj = -1; }
         ++re;
         ne = re < np ? base_c + slot_of(re, tau_c, k_c) + tau_c : static_cast<i64>(NEVER) * 2;
       }
@@ -185,11 +186,12 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         np = w;
         tau_c = sh.tau[ph]; k_c = sh.k[ph]; base_c = sh.pbase[ph];
         rs = 0; re = 0; ns = base_c; ne = base_c + tau_c;
-        fpos = 0;
+        fpos = 0; cj = -1;
       }
       // (2) pipeline runs that start now
       bool dropped = false;
       while (ns <= t) {
+        cj = -1;                                        // the job that starts may be the known candidate
         const int j = list[rs];
         const int oj = O[j], sj = S[j];
         const int len = oj < static_cast<int>(tau_c) ? oj : static_cast<int>(tau_c);
@@ -218,6 +220,27 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         ns = rs < np ? base_c + slot_of(rs, tau_c, k_c) : static_cast<i64>(NEVER) * 2;
       }
       if (t == H) break;                                // nothing runs in round H; only completions were due
+      if (left == 0) {
+        // Every job is done, so every run the pipeline has yet to start is dropped: what is left of the plan are
+        // the runs in progress, which are completing runs of ranks between the two cursors (a killed run in
+        // progress would belong to an unfinished job).  A run in progress ends at be > t and began at be - o.
+        __syncwarp();
+        for (int u = t + lane; u < H; u += 32) prof[u] = 0;
+        __syncwarp();
+        for (int r = re; r < rs; ++r) {
+          const int j = list[r];
+          const int end = be[j];
+          if (end > t) {
+            const int first = end - O[j], sj = S[j];
+            for (int u = t + lane; u < end; u += 32) prof[u] += sj + (u - first) + 1;
+            __syncwarp();
+          }
+        }
+        i64 pk = 0;
+        for (int u = t + lane; u < hmax; u += 32) pk = max_i64(pk, prof[u]);
+        peak = max_i64(peak, warp_max(pk));
+        break;
+      }
       if ((t & 31) == 0 || dropped) {
         __syncwarp();
         const int u = (t & ~31) + lane;
@@ -243,22 +266,25 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         __syncwarp();
         int a = 0, b = np;                              // its position in the list (ascending job indices)
         while (a < b) { const int m = (a + b) >> 1; if (list[m] < j) a = m + 1; else b = m; }
-        fpos = min(fpos, a);
+        if (a < fpos) { fpos = a; cj = -1; }
       }
       // (4) first come first served
       for (;;) {
-        int c = -1;
-        while (fpos < np) {
-          const int q = fpos + lane;
-          bool fr = false;
-          if (q < np) { const int j = list[q]; fr = !done[j] && sst[j] < 0 && be[j] <= t; }
-          const unsigned hit = __ballot_sync(0xffffffffu, fr);
-          if (hit) { fpos += __ffs(static_cast<int>(hit)) - 1; c = fpos; break; }
-          fpos += 32;
+        if (cj == -1) {                                 // look for the lowest free job at or after fpos
+          int c = -1;
+          while (fpos < np) {
+            const int q = fpos + lane;
+            bool fr = false;
+            if (q < np) { const int j = list[q]; fr = !done[j] && sst[j] < 0 && be[j] <= t; }
+            const unsigned hit = __ballot_sync(0xffffffffu, fr);
+            if (hit) { fpos += __ffs(static_cast<int>(hit)) - 1; c = fpos; break; }
+            fpos += 32;
+          }
+          if (c < 0) { fpos = np; cj = -2; } else { cj = list[c]; cs = S[cj]; }
         }
-        if (c < 0) { fpos = np; break; }
-        const int j = list[c];
-        const int sc = S[j];
+        if (cj < 0) break;
+        const int j = cj;
+        const int sc = cs;
         if (B + A + static_cast<i64>(t) * cnt + sc + 1 > M) break;
         if (top == static_cast<int>(cap)) {             // stale entries fill the stack: keep the live ones, in order
           int w = 0;
@@ -282,7 +308,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         A += static_cast<i64>(sc) + 1 - t;
         ++cnt;
         next_comp = min(next_comp, t + O[j]);
-        ++fpos;
+        ++fpos; cj = -1;
       }
       // (5) the round's memory
       const i64 mem = B + A + static_cast<i64>(t) * cnt;

@@ -44,7 +44,7 @@ def _bench_call(par, name, n_inst):
     first = Scheduler.scalars(P, dev)
     ctx.build_schedule(inst, settings, dict(n_runs=torch.zeros(P, dtype=torch.int64, device=dev)), first,
                        window=window, max_jobs=n)
-    geo = torch.from_numpy(settings["family"] <= 1).to(dev)
+    geo = torch.from_numpy(np.array([bench.stores_profile(name, int(f)) for f in settings["family"]])).to(dev)
     cap = torch.where(geo, first["horizon"], torch.zeros_like(first["horizon"]))
     poff = torch.zeros(P + 1, dtype=torch.int64, device=dev)
     poff[1:] = torch.cumsum(cap, 0)
@@ -126,6 +126,21 @@ def test_config2_full_size_stratified(par, pool):
     budgets = {(int(settings[e]["M"]), int(settings[e]["family"])) for e in sample}
     assert len(sample) == 256 and len(budgets) == 16
     _check_sample(pool, inst, settings, window, n, out, ev, sample, "config 2")
+
+
+@pytest.mark.parametrize("name", ["c2d", "c2s"])
+def test_config2_refill_and_speculation_full_size_stratified(par, pool, name):
+    """Config 2's 1,024 instances x 8 budgets under the dynamic refill / under speculative runs, one call as
+    bench.py times it; 8 instances under every budget compared in full (64 evaluations), the rest by properties
+    (every job completes, completion = start + o for the run that completed it, every round fits)."""
+    inst, settings, window, n, out, ev, first = _bench_call(par, name, 1024)
+    _check_properties(settings, n, out, ev, inst)
+    assert bool((ev["horizon"] <= first["horizon"]).all()) and bool((ev["flow"] <= first["flow"]).all())
+    rng = np.random.default_rng(22)
+    chosen = set(int(i) for i in rng.choice(1024, 8, replace=False))
+    sample = [e for e in range(settings.shape[0]) if int(settings[e]["instance"]) in chosen]
+    assert len(sample) == 64 and len({int(settings[e]["M"]) for e in sample}) == 8
+    _check_sample(pool, inst, settings, window, n, out, ev, sample, name)
 
 
 def test_config5_full_size_stratified(par, pool):
