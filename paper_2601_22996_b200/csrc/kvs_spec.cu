@@ -47,8 +47,8 @@ __device__ __forceinline__ i64 slot_of(int r, u32 tau, u32 k) {
 __device__ __forceinline__ int warp_min_int(int v) { return -warp_max(-v); }
 
 // Bytes of one warp's working storage for instances of at most n jobs: five int arrays (end of the latest
-// pipeline run, start of the speculative run or -1, stack of speculative runs as job and start, participant
-// list) and two byte arrays (class, done flag).
+// pipeline run, start of the speculative run or -1, stack of speculative runs as job and completion round,
+// participant list) and two byte arrays (class, done flag).
 __host__ __device__ inline i64 spec_stride(i64 n) { return (22 * n + 255) & ~static_cast<i64>(255); }
 
 __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
@@ -63,8 +63,8 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
   int* const be = reinterpret_cast<int*>(mine);
   int* const sst = be + cap;
   int* const stk_job = sst + cap;
-  int* const stk_start = stk_job + cap;
-  int* const list = stk_start + cap;
+  int* const stk_fin = stk_job + cap;                    // round in which the entry's run would complete
+  int* const list = stk_fin + cap;
   unsigned char* const cls = reinterpret_cast<unsigned char*>(list + cap);
   unsigned char* const done = cls + cap;
 
@@ -136,26 +136,32 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
       // (1) speculative completions
       if (t == next_comp) {
         int nc = NEVER;
-        for (int q0 = 0; q0 < top; q0 += 32) {
-          const int q = q0 + lane;
-          bool fin = false;
-          int j = 0, s0 = 0;
-          if (q < top) {
-            j = stk_job[q]; s0 = stk_start[q];
-            if (sst[j] == s0) {                         // a live entry
-              const int f = s0 + O[j];
-              if (f == t) fin = true; else nc = min(nc, f);
+        for (int g0 = 0; g0 < top; g0 += 128) {         // four chunks' completion rounds are loaded together
+          int fq[4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) fq[c] = g0 + 32 * c + lane < top ? stk_fin[g0 + 32 * c + lane] : NEVER;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int q = g0 + 32 * c + lane;
+            const int f = fq[c];
+            if (f > t) nc = min(nc, f);                 // stale entries included: they cost one empty scan at most
+            if (__ballot_sync(0xffffffffu, f == t) == 0) continue;
+            bool fin = false;
+            int j = 0, s0 = 0;
+            if (f == t) {
+              j = stk_job[q]; s0 = t - O[j];
+              fin = sst[j] == s0;                       // a live entry
             }
-          }
-          const unsigned fm = __ballot_sync(0xffffffffu, fin);
-          if (fm) {
-            if (fin) { done[j] = 1; sst[j] = -1; js[j] = s0; jc[j] = t; }
-            const i64 dA = warp_sum(fin ? static_cast<i64>(S[j]) + 1 - s0 : static_cast<i64>(0));
-            const i64 dS = warp_sum(fin ? static_cast<i64>(O[j]) : static_cast<i64>(0));
-            const int kf = __popc(fm);
-            A -= dA; steps += dS; flow += static_cast<i64>(kf) * t;
-            cnt -= kf; left -= kf; runs += kf;
-            hmax = max(hmax, t);
+            const unsigned fm = __ballot_sync(0xffffffffu, fin);
+            if (fm) {
+              if (fin) { done[j] = 1; sst[j] = -1; js[j] = s0; jc[j] = t; }
+              const i64 dA = warp_sum(fin ? static_cast<i64>(S[j]) + 1 - s0 : static_cast<i64>(0));
+              const i64 dS = warp_sum(fin ? static_cast<i64>(O[j]) : static_cast<i64>(0));
+              const int kf = __popc(fm);
+              A -= dA; steps += dS; flow += static_cast<i64>(kf) * t;
+              cnt -= kf; left -= kf; runs += kf;
+              hmax = max(hmax, t);
+            }
           }
         }
         next_comp = warp_min_int(nc);
@@ -163,8 +169,10 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
       }
       // slots that have ended: a job killed at the end of its slot is free again
       while (ne <= t) {
-        const int j = list[re];
-        if (!done[j] && sst[j] < 0 && re < fpos) { fpos = re; cj = -1; }
+        if (re < fpos) {                                // else it cannot lower the position
+          const int j = list[re];
+          if (!done[j] && sst[j] < 0) { fpos = re; cj = -1; }
+        }
         ++re;
         ne = re < np ? base_c + slot_of(re, tau_c, k_c) + tau_c : static_cast<i64>(NEVER) * 2;
       }
@@ -253,7 +261,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         while (top > 0) {                               // the live entry nearest to the top
           --top;
           const int jj = stk_job[top];
-          s0 = stk_start[top];
+          s0 = stk_fin[top] - O[jj];
           if (sst[jj] == s0) { j = jj; break; }
         }
         if (j < 0) break;
@@ -264,9 +272,11 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         runs += t > s0 ? 1 : 0;
         if (lane == 0) sst[j] = -1;
         __syncwarp();
-        int a = 0, b = np;                              // its position in the list (ascending job indices)
-        while (a < b) { const int m = (a + b) >> 1; if (list[m] < j) a = m + 1; else b = m; }
-        if (a < fpos) { fpos = a; cj = -1; }
+        if (cj < 0 || j < cj) {                         // it may come before the known candidate
+          int a = 0, b = np;                            // its position in the list (ascending job indices)
+          while (a < b) { const int m = (a + b) >> 1; if (list[m] < j) a = m + 1; else b = m; }
+          if (a < fpos) { fpos = a; cj = -1; }
+        }
       }
       // (4) first come first served
       for (;;) {
@@ -286,28 +296,29 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         const int j = cj;
         const int sc = cs;
         if (B + A + static_cast<i64>(t) * cnt + sc + 1 > M) break;
-        if (top == static_cast<int>(cap)) {             // stale entries fill the stack: keep the live ones, in order
+        if (top == static_cast<int>(cap) || top > 2 * cnt + 64) {   // mostly stale entries: keep the live ones, in order
           int w = 0;
           for (int q0 = 0; q0 < top; q0 += 32) {
             const int q = q0 + lane;
             bool live = false;
-            int jj = 0, s0 = 0;
-            if (q < top) { jj = stk_job[q]; s0 = stk_start[q]; live = sst[jj] == s0; }
+            int jj = 0, ff = 0;
+            if (q < top) { jj = stk_job[q]; ff = stk_fin[q]; live = sst[jj] == ff - O[jj]; }
             const unsigned m = __ballot_sync(0xffffffffu, live);
             __syncwarp();
-            if (live) { const int d = w + __popc(m & lt_mask); stk_job[d] = jj; stk_start[d] = s0; }
+            if (live) { const int d = w + __popc(m & lt_mask); stk_job[d] = jj; stk_fin[d] = ff; }
             w += __popc(m);
             __syncwarp();
           }
           top = w;
         }
         __syncwarp();
-        if (lane == 0) { sst[j] = t; stk_job[top] = j; stk_start[top] = t; }
+        const int fin = t + O[j];
+        if (lane == 0) { sst[j] = t; stk_job[top] = j; stk_fin[top] = fin; }
         __syncwarp();
         ++top;
         A += static_cast<i64>(sc) + 1 - t;
         ++cnt;
-        next_comp = min(next_comp, t + O[j]);
+        next_comp = min(next_comp, fin);
         ++fpos; cj = -1;
       }
       // (5) the round's memory
