@@ -24,6 +24,7 @@
 // final memory(t) is exact whenever it is below 2^32, which a per-phase bound guarantees
 // (otherwise the evaluation reports KVS_EVAL_RANGE and skips the profile).
 #include "kvs_events.cuh"
+#include "kvs_ladder.cuh"
 
 namespace {
 
@@ -35,23 +36,6 @@ constexpr int RPT = 4;                     // consecutive ranks per thread in th
 constexpr int CHUNK = T * RPT;
 constexpr int VEC = ITEMS / 4;              // 16-byte vectors per thread and tile
 static_assert(ITEMS % 4 == 0 && (ITEMS & (ITEMS - 1)) == 0, "rounds per thread: a power of two, whole vectors");
-
-typedef unsigned __int128 u128;
-
-__device__ __forceinline__ i64 gcd_i64(i64 x, i64 y) {
-  while (y) { i64 t = x % y; x = y; y = t; }
-  return x;
-}
-
-// Largest k >= 1 with s*k + (tau*k + tau + k - gcd(tau, k))/2 <= M, given s + tau <= M.
-// The condition reads k*(2s+tau+1) <= 2M - tau + gcd(tau,k); because 1 <= gcd <= tau the answer
-// is k0 or k0 + 1 with k0 = floor((2M - tau + 1) / (2s + tau + 1)).
-__device__ i64 max_parallelism(i64 tau, i64 s, i64 M) {
-  const i64 D = 2 * s + tau + 1;
-  const i64 k0 = (2 * M - tau + 1) / D;
-  const i64 k1 = k0 + 1;
-  return (k1 * D <= 2 * M - tau + gcd_i64(tau, k1)) ? k1 : k0;
-}
 
 // Shared-memory word of round e of a tile.  Thread t owns rounds ITEMS*t .. ITEMS*t + ITEMS-1 as VEC
 // 4-word vectors; vector c of thread t sits at vector index c*T + t, so a warp's vector access is
@@ -99,51 +83,11 @@ __device__ __forceinline__ void add_event(u32* dA, u32* dB, int idx, u32 c, u32 
 // max-parallelism), or the batch size of the simultaneous schedule; 0 if not even one job fits.
 __device__ __forceinline__ i64 phase_parallelism(i64 tau, i64 s, i64 M, bool batches) {
   if (s + tau > M) return 0;
-  return batches ? M / (s + tau) : max_parallelism(tau, s, M);
+  return batches ? M / (s + tau) : max_parallelism64(tau, s, M);
 }
 
 __device__ void build_ladder(Shared& sh, i64 X, int a, int b, i64 beta0, i64 s_bar, i64 M, bool batches) {
-  const int lane = lane_id();
-  if (beta0 <= 0) {
-    if (lane == 0) {
-      // ell = largest j with a^j <= X * b^j, powers kept exactly in 128 bits
-      u128 pa = 1, pb = 1;
-      int ell = 0;
-      sh.pw_a[0] = 1; sh.pw_b[0] = 1;
-      while (ell + 1 < KVS_MAX_PHASES + 1) {
-        const u128 na = pa * static_cast<u128>(a), nb = pb * static_cast<u128>(b);
-        if (na > static_cast<u128>(X) * nb) break;
-        pa = na; pb = nb; ++ell;
-        sh.pw_a[ell] = pa; sh.pw_b[ell] = pb;
-      }
-      sh.n_phases = (ell + 1 <= KVS_MAX_PHASES) ? ell + 1 : 0;
-    }
-    __syncwarp();
-    const int L = sh.n_phases;
-    for (int p = lane; p < L; p += 32) {
-      const int j = L - 1 - p;  // tau_p = floor(X * b^j / a^j)
-      const i64 t = (a == 2 && b == 1) ? (X >> j) : static_cast<i64>(static_cast<u128>(X) * sh.pw_b[j] / sh.pw_a[j]);
-      sh.tau[p] = t;
-      sh.k[p] = phase_parallelism(t, s_bar, M, batches);
-    }
-  } else {
-    if (lane == 0) {
-      u128 pa = 1, pb = 1;
-      int p = 0;
-      for (;; ++p) {
-        if (p >= KVS_MAX_PHASES) { p = -1; break; }
-        // tau_p = min(floor(beta0 * a^p / b^p), X)
-        const u128 num = static_cast<u128>(beta0) * pa;
-        i64 t = (num >= static_cast<u128>(X) * pb) ? X : static_cast<i64>(num / pb);
-        sh.tau[p] = t;
-        sh.k[p] = phase_parallelism(t, s_bar, M, batches);
-        if (t >= X) break;
-        pa *= static_cast<u128>(a); pb *= static_cast<u128>(b);
-      }
-      sh.n_phases = p + 1;
-    }
-  }
-  __syncwarp();
+  ladder_phases(sh, X, a, b, beta0, [=](i64 t) { return phase_parallelism(t, s_bar, M, batches); });
 }
 
 // Exclusive block scan of a small per-thread count; returns this thread's offset, total in *total.
@@ -644,7 +588,7 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, KVS_EVAL_MIN_CTAS) k_build_e
       } else if (tid == 0) {
         i64 tau = st.tau > 0 ? st.tau : static_cast<i64>(KEY[seg_hi - 1]);  // largest key of the segment
         i64 k = st.k;
-        if (k <= 0) k = simultaneous ? M / (s_bar + tau) : (s_bar + tau <= M ? max_parallelism(tau, s_bar, M) : 0);
+        if (k <= 0) k = simultaneous ? M / (s_bar + tau) : (s_bar + tau <= M ? max_parallelism64(tau, s_bar, M) : 0);
         sh.tau[0] = tau; sh.k[0] = k;
         sh.ent[0] = 0; sh.ent[1] = nseg;
       }

@@ -1,6 +1,6 @@
 // Geometric ladder of slice lengths and the largest memory-feasible parallelism of each slice (first
 // line of the two geometric algorithms; Lemma "Peak Memory Usage of SPS"; Eq. max-parallelism), and
-// the class of a response length.  Shared by the fast fused kernel and the bound kernel.
+// the class of a response length.  Shared by the fused kernels, the bound kernel and the speculative-run kernel.
 #pragma once
 
 #include "kvs_internal.cuh"
@@ -27,13 +27,29 @@ __device__ inline u32 max_parallelism32(u32 tau, u32 s, u32 M) {
   return (k1 * D <= 2ull * M - tau + gcd_u32(tau, static_cast<u32>(k1))) ? static_cast<u32>(k1) : static_cast<u32>(k0);
 }
 
-// `sh` provides pw_a, pw_b (u128 [MAXP + 1]), tau, k (u32 [MAXP]) and n_phases; called by one warp.
-template <class Sh>
-__device__ void ladder32(Sh& sh, i64 X, int a, int b, i64 beta0, u32 s_bar, u32 M) {
+// The same in 64-bit arithmetic (the general kernel: budgets and slices up to 2^31, carried in int64).
+__device__ __forceinline__ i64 gcd_i64(i64 x, i64 y) {
+  while (y) { const i64 t = x % y; x = y; y = t; }
+  return x;
+}
+__device__ inline i64 max_parallelism64(i64 tau, i64 s, i64 M) {
+  const i64 D = 2 * s + tau + 1;
+  const i64 k0 = (2 * M - tau + 1) / D;
+  const i64 k1 = k0 + 1;
+  return (k1 * D <= 2 * M - tau + gcd_i64(tau, k1)) ? k1 : k0;
+}
+
+// The ladder tau_0 .. tau_(L-1) of one evaluation and, through `par(tau)`, the parallelism of every slice.
+// `sh` provides pw_a, pw_b (u128 [MAXP + 1]), tau, k ([MAXP], 32- or 64-bit) and n_phases (0 = the ladder
+// needs more than MAXP slices); called by one warp.
+template <class Sh, class Par>
+__device__ __forceinline__ void ladder_phases(Sh& sh, i64 X, int a, int b, i64 beta0, Par par) {
   constexpr int MAXP = KVS_MAX_PHASES;
+  typedef decltype(sh.tau[0] + 0) V;                      // value type of the tables
   const int lane = lane_id();
   if (beta0 <= 0) {
     if (lane == 0) {
+      // ell = largest j with a^j <= X * b^j, powers kept exactly in 128 bits
       u128 pa = 1, pb = 1;
       int ell = 0;
       sh.pw_a[0] = 1; sh.pw_b[0] = 1;
@@ -49,10 +65,10 @@ __device__ void ladder32(Sh& sh, i64 X, int a, int b, i64 beta0, u32 s_bar, u32 
     const int L = sh.n_phases;
     for (int p = lane; p < L; p += 32) {
       const int j = L - 1 - p;  // tau_p = floor(X * b^j / a^j)
-      const u32 t = (a == 2 && b == 1) ? static_cast<u32>(X >> j)
-                                       : static_cast<u32>(static_cast<u128>(X) * sh.pw_b[j] / sh.pw_a[j]);
+      const V t = (a == 2 && b == 1) ? static_cast<V>(X >> j)
+                                     : static_cast<V>(static_cast<u128>(X) * sh.pw_b[j] / sh.pw_a[j]);
       sh.tau[p] = t;
-      sh.k[p] = max_parallelism32(t, s_bar, M);
+      sh.k[p] = par(t);
     }
   } else {
     if (lane == 0) {
@@ -61,16 +77,22 @@ __device__ void ladder32(Sh& sh, i64 X, int a, int b, i64 beta0, u32 s_bar, u32 
       for (;; ++p) {
         if (p >= MAXP) { p = -1; break; }
         const u128 num = static_cast<u128>(beta0) * pa;   // tau_p = min(floor(beta0 * a^p / b^p), X)
-        const u32 t = (num >= static_cast<u128>(X) * pb) ? static_cast<u32>(X) : static_cast<u32>(num / pb);
+        const V t = (num >= static_cast<u128>(X) * pb) ? static_cast<V>(X) : static_cast<V>(num / pb);
         sh.tau[p] = t;
-        sh.k[p] = max_parallelism32(t, s_bar, M);
-        if (t >= X) break;
+        sh.k[p] = par(t);
+        if (static_cast<i64>(t) >= X) break;
         pa *= static_cast<u128>(a); pb *= static_cast<u128>(b);
       }
       sh.n_phases = p + 1;
     }
   }
   __syncwarp();
+}
+
+// 32-bit tables with the largest memory-feasible parallelism of the staggered pipeline.
+template <class Sh>
+__device__ __forceinline__ void ladder32(Sh& sh, i64 X, int a, int b, i64 beta0, u32 s_bar, u32 M) {
+  ladder_phases(sh, X, a, b, beta0, [=](u32 t) { return max_parallelism32(t, s_bar, M); });
 }
 
 // class(v) = first p with tau_p >= v (tau is nondecreasing and tau_(L-1) >= v)

@@ -19,8 +19,8 @@
 // The speculative runs hold A + t * count tokens in round t (a run started at t0 holds s + 1 - t0 + t).
 // Per phase the participants are kept as a list in index order, so that rank r is entry r.  Two cursors walk
 // it: one over the run starts, one over the slot ends start + tau (nondecreasing in the rank), which is when a
-// killed job becomes free to speculate.  `fpos` is a position such that no entry before it is free at the
-// moment; the events that free a job (a slot end, a kill for memory) lower it.
+// killed job becomes free to speculate.  No entry before position `fpos` and none at or after `fhi` is free at the
+// moment; the events that free a job (a slot end, a kill for memory) widen that range, a scan narrows it.
 #include "kvs_ladder.cuh"
 
 namespace {
@@ -46,8 +46,15 @@ __device__ __forceinline__ i64 slot_of(int r, u32 tau, u32 k) {
 
 __device__ __forceinline__ int warp_min_int(int v) { return -warp_max(-v); }
 
-// Bytes of one warp's working storage for instances of at most n jobs: five int arrays (end of the latest
-// pipeline run, start of the speculative run or -1, stack of speculative runs as job and completion round,
+// Number of ranks r < np with floor(r * tau / k) <= x: r * tau < (x + 1) * k, so ceil((x + 1) * k / tau) of them.
+__device__ __forceinline__ int started(i64 x, u32 tau, u32 k, int np) {
+  if (x < 0) return 0;
+  const u64 v = (static_cast<u64>(x + 1) * k + tau - 1) / tau;
+  return v < static_cast<u64>(np) ? static_cast<int>(v) : np;
+}
+
+// Bytes of one warp's working storage for instances of at most n jobs: five int arrays (position in the phase's
+// list, start of the speculative run or -1, stack of speculative runs as job and completion round,
 // participant list) and two byte arrays (class, done flag).
 __host__ __device__ inline i64 spec_stride(i64 n) { return (22 * n + 255) & ~static_cast<i64>(255); }
 
@@ -60,8 +67,8 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
   if (wslot >= p.n_warps) return;
   const i64 cap = p.max_jobs;
   unsigned char* const mine = p.scratch + wslot * spec_stride(cap);
-  int* const be = reinterpret_cast<int*>(mine);
-  int* const sst = be + cap;
+  int* const pos_of = reinterpret_cast<int*>(mine);    // position of a job in the current phase's list
+  int* const sst = pos_of + cap;
   int* const stk_job = sst + cap;
   int* const stk_fin = stk_job + cap;                    // round in which the entry's run would complete
   int* const list = stk_fin + cap;
@@ -100,7 +107,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
       const u32 oi = static_cast<u32>(O[i]);
       const int c = pow2 ? class_pow2(static_cast<u32>(X), oi) : class_of(sh.tau, L, oi);
       cls[i] = static_cast<unsigned char>(c);
-      done[i] = 0; be[i] = 0; sst[i] = -1; list[i] = i;
+      done[i] = 0; pos_of[i] = i; sst[i] = -1; list[i] = i;
       atomicAdd(&sh.hist[c], 1u);
     }
     __syncwarp();
@@ -126,7 +133,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
     i64 A = 0;                                          // speculative runs hold A + t * cnt tokens in round t
     int cnt = 0, top = 0;                               // running speculative runs; entries on the stack (some stale)
     int next_comp = NEVER;                              // no speculative run completes before this round
-    int fpos = 0;
+    int fpos = 0, fhi = n;
     int cj = -1, cs = 0;                                // the free job at fpos and its prompt length, while known (cj = -2: none is free)
     int left = n;
     i64 flow = 0, steps = 0, runs = 0, peak = 0;
@@ -167,13 +174,22 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         next_comp = warp_min_int(nc);
         __syncwarp();
       }
-      // slots that have ended: a job killed at the end of its slot is free again
-      while (ne <= t) {
-        if (re < fpos) {                                // else it cannot lower the position
-          const int j = list[re];
-          if (!done[j] && sst[j] < 0) { fpos = re; cj = -1; }
+      // slots that have ended: a job killed at the end of its slot is free again.  The ranks whose slots end by
+      // round t are [re, started(t - tau)); only those before fpos can lower it.
+      if (ne <= t) {
+        const int eend = started(static_cast<i64>(t) - tau_c - base_c, tau_c, k_c, np);
+        // the ranks [re, eend) are free now unless done or running speculatively; those before fpos are looked at
+        // here (the known candidate stays the lowest free job if none of them is), the others lie in the range
+        const int lim = min(eend, fpos);
+        for (int r0 = re; r0 < lim; r0 += 32) {
+          const int r = r0 + lane;
+          bool fr = false;
+          if (r < lim) { const int j = list[r]; fr = !done[j] && sst[j] < 0; }
+          const unsigned hit = __ballot_sync(0xffffffffu, fr);
+          if (hit) { fpos = r0 + __ffs(static_cast<int>(hit)) - 1; cj = -1; break; }
         }
-        ++re;
+        if (eend > fhi && (cj == -1 || eend > lim)) fhi = eend;
+        re = eend;
         ne = re < np ? base_c + slot_of(re, tau_c, k_c) + tau_c : static_cast<i64>(NEVER) * 2;
       }
       // the next phase begins: its participants are the jobs of a later class, in index order
@@ -187,57 +203,92 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
           if (q < np) { j = list[q]; keep = cls[j] >= ph; }
           const unsigned m = __ballot_sync(0xffffffffu, keep);
           __syncwarp();
-          if (keep) list[w + __popc(m & lt_mask)] = j;
+          if (keep) { const int d = w + __popc(m & lt_mask); list[d] = j; pos_of[j] = d; }
           w += __popc(m);
           __syncwarp();
         }
         np = w;
         tau_c = sh.tau[ph]; k_c = sh.k[ph]; base_c = sh.pbase[ph];
         rs = 0; re = 0; ns = base_c; ne = base_c + tau_c;
-        fpos = 0; cj = -1;
+        fpos = 0; fhi = np; cj = -1;
       }
-      // (2) pipeline runs that start now
-      bool dropped = false;
-      while (ns <= t) {
-        cj = -1;                                        // the job that starts may be the known candidate
-        const int j = list[rs];
-        const int oj = O[j], sj = S[j];
-        const int len = oj < static_cast<int>(tau_c) ? oj : static_cast<int>(tau_c);
-        if (done[j]) {
-          for (int u = lane; u < len; u += 32) prof[t + u] -= sj + u + 1;     // dropped from the plan
-          dropped = true;
-        } else {
-          const int s0 = sst[j];
-          __syncwarp();
-          if (s0 >= 0) {                                // its speculative run is killed; the stack entry goes stale
-            A -= static_cast<i64>(sj) + 1 - s0;
-            --cnt;
-            steps += t - s0;
-            runs += t > s0 ? 1 : 0;
+      // (2) pipeline runs that start now: ranks [rs, started(t)), 32 at a time (they concern different jobs)
+      if (ns <= t) {
+        const int rend = started(static_cast<i64>(t) - base_c, tau_c, k_c, np);
+        bool cand_started = false;                      // a job that starts may be the known candidate
+        for (int r0 = rs; r0 < rend; r0 += 32) {
+          const int r = r0 + lane;
+          const bool act = r < rend;
+          int j = 0, oj = 0, sj = 0, s0 = -1;
+          bool dn = false;
+          if (act) { j = list[r]; oj = O[j]; sj = S[j]; dn = done[j] != 0; s0 = sst[j]; }
+          if (cj >= 0 && __ballot_sync(0xffffffffu, act && j == cj)) cand_started = true;
+          const int len = oj < static_cast<int>(tau_c) ? oj : static_cast<int>(tau_c);
+          const bool run = act && !dn, drop = act && dn;
+          const bool kill = run && s0 >= 0;             // its speculative run is killed; the stack entry goes stale
+          const bool comp = run && len == oj;
+          const unsigned km = __ballot_sync(0xffffffffu, kill);
+          if (km) {
+            A -= warp_sum(kill ? static_cast<i64>(sj) + 1 - s0 : static_cast<i64>(0));
+            steps += warp_sum(kill ? static_cast<i64>(t - s0) : static_cast<i64>(0));
+            cnt -= __popc(km);
+            runs += __popc(__ballot_sync(0xffffffffu, kill && t > s0));
           }
-          steps += len; ++runs;
-          if (lane == 0) {
-            sst[j] = -1;
-            be[j] = t + len;
-            if (len == oj) { done[j] = 1; js[j] = t; jc[j] = t + len; }
+          const unsigned rm = __ballot_sync(0xffffffffu, run);
+          if (rm) {
+            steps += warp_sum(run ? static_cast<i64>(len) : static_cast<i64>(0));
+            runs += __popc(rm);
+            if (run) {
+              sst[j] = -1;
+              if (comp) { done[j] = 1; js[j] = t; jc[j] = t + len; }
+            }
+            const unsigned cm = __ballot_sync(0xffffffffu, comp);
+            if (cm) {
+              left -= __popc(cm);
+              flow += warp_sum(comp ? static_cast<i64>(t + len) : static_cast<i64>(0));
+              hmax = max(hmax, warp_max(comp ? t + len : 0));
+            }
           }
-          if (len == oj) { --left; flow += t + len; hmax = max(hmax, t + len); }
-          __syncwarp();
+          // dropped from the plan: short ramps lane by lane, long ones by the whole warp; the rounds of the
+          // window held in registers are corrected there (the round of lane l is t - (t & 31) + l)
+          unsigned dm = __ballot_sync(0xffffffffu, drop);
+          if (dm) {
+            if (drop && len <= 64)
+              for (int u = 0; u < len; ++u) atomicSub(&prof[t + u], sj + u + 1);
+            unsigned lm = __ballot_sync(0xffffffffu, drop && len > 64);
+            while (lm) {
+              const int src = __ffs(static_cast<int>(lm)) - 1;
+              lm &= lm - 1u;
+              const int ls = __shfl_sync(0xffffffffu, len, src), ss = __shfl_sync(0xffffffffu, sj, src);
+              for (int u = lane; u < ls; u += 32) atomicSub(&prof[t + u], ss + u + 1);
+            }
+            if ((t & 31) != 0) {                        // at a window's first round the window is loaded afterwards
+              const int u = lane - (t & 31);            // this lane's round, counted from t
+              while (dm) {
+                const int src = __ffs(static_cast<int>(dm)) - 1;
+                dm &= dm - 1u;
+                const int ls = __shfl_sync(0xffffffffu, len, src), ss = __shfl_sync(0xffffffffu, sj, src);
+                if (u >= 0 && u < ls) Bw -= ss + u + 1;
+              }
+            }
+          }
         }
-        ++rs;
+        __syncwarp();
+        if (cand_started) cj = -1;
+        rs = rend;
         ns = rs < np ? base_c + slot_of(rs, tau_c, k_c) : static_cast<i64>(NEVER) * 2;
       }
       if (t == H) break;                                // nothing runs in round H; only completions were due
       if (left == 0) {
         // Every job is done, so every run the pipeline has yet to start is dropped: what is left of the plan are
         // the runs in progress, which are completing runs of ranks between the two cursors (a killed run in
-        // progress would belong to an unfinished job).  A run in progress ends at be > t and began at be - o.
+        // progress would belong to an unfinished job).  Such a run's completion round lies beyond t and it began o earlier.
         __syncwarp();
         for (int u = t + lane; u < H; u += 32) prof[u] = 0;
         __syncwarp();
         for (int r = re; r < rs; ++r) {
           const int j = list[r];
-          const int end = be[j];
+          const int end = jc[j];                        // beyond t only for a completing run of the pipeline in progress
           if (end > t) {
             const int first = end - O[j], sj = S[j];
             for (int u = t + lane; u < end; u += 32) prof[u] += sj + (u - first) + 1;
@@ -245,14 +296,14 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
           }
         }
         i64 pk = 0;
-        for (int u = t + lane; u < hmax; u += 32) pk = max_i64(pk, prof[u]);
+        for (int u = t + lane; u < hmax; u += 32) pk = max_i64(pk, __ldcg(prof + u));
         peak = max_i64(peak, warp_max(pk));
         break;
       }
-      if ((t & 31) == 0 || dropped) {
+      if ((t & 31) == 0) {                              // the plan's next 32 rounds, past the first-level cache: other lanes' atomics wrote them
         __syncwarp();
-        const int u = (t & ~31) + lane;
-        Bw = u < H ? prof[u] : 0;
+        const int u = t + lane;
+        Bw = u < H ? __ldcg(prof + u) : 0;
       }
       const i64 B = __shfl_sync(0xffffffffu, Bw, t & 31);
       // (3) the pipeline comes first
@@ -272,54 +323,70 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         runs += t > s0 ? 1 : 0;
         if (lane == 0) sst[j] = -1;
         __syncwarp();
-        if (cj < 0 || j < cj) {                         // it may come before the known candidate
-          int a = 0, b = np;                            // its position in the list (ascending job indices)
-          while (a < b) { const int m = (a + b) >> 1; if (list[m] < j) a = m + 1; else b = m; }
-          if (a < fpos) { fpos = a; cj = -1; }
-        }
+        const int a = pos_of[j];                        // free again: it may come before the known candidate
+        if (a < fpos) { fpos = a; cj = -1; }
+        if (a >= fhi) { fhi = a + 1; if (cj == -2) cj = -1; }
       }
-      // (4) first come first served
+      // (4) first come first served: the free jobs of a window of 32 list entries are admitted together as far as
+      // their first rounds fit, in order; the first that does not fit ends the round's admissions
       for (;;) {
-        if (cj == -1) {                                 // look for the lowest free job at or after fpos
-          int c = -1;
-          while (fpos < np) {
-            const int q = fpos + lane;
-            bool fr = false;
-            if (q < np) { const int j = list[q]; fr = !done[j] && sst[j] < 0 && be[j] <= t; }
-            const unsigned hit = __ballot_sync(0xffffffffu, fr);
-            if (hit) { fpos += __ffs(static_cast<int>(hit)) - 1; c = fpos; break; }
-            fpos += 32;
-          }
-          if (c < 0) { fpos = np; cj = -2; } else { cj = list[c]; cs = S[cj]; }
+        const i64 room = M - (B + A + static_cast<i64>(t) * cnt);
+        if (cj == -2 || (cj >= 0 && cs + 1 > room) || room <= 0) break;
+        // the jobs in a pipeline run are the ranks whose slot has begun and not ended: [re, rs)
+        if (fpos >= re && fpos < rs) fpos = rs;
+        if (fpos >= fhi) { fpos = np; fhi = 0; cj = -2; break; }
+        const int q = fpos + lane;
+        bool fr = false;
+        int j = 0, sj = 0;
+        if (q < fhi && !(q >= re && q < rs)) { j = list[q]; fr = !done[j] && sst[j] < 0; }
+        const unsigned hit = __ballot_sync(0xffffffffu, fr);
+        if (!hit) { fpos += 32; cj = -1; continue; }
+        if (fr) sj = S[j];
+        i64 need = fr ? static_cast<i64>(sj) + 1 : 0;   // inclusive prefix sums over the window, in list order
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const i64 y = __shfl_up_sync(0xffffffffu, need, d);
+          if (lane >= d) need += y;
         }
-        if (cj < 0) break;
-        const int j = cj;
-        const int sc = cs;
-        if (B + A + static_cast<i64>(t) * cnt + sc + 1 > M) break;
-        if (top == static_cast<int>(cap) || top > 2 * cnt + 64) {   // mostly stale entries: keep the live ones, in order
-          int w = 0;
-          for (int q0 = 0; q0 < top; q0 += 32) {
-            const int q = q0 + lane;
-            bool live = false;
-            int jj = 0, ff = 0;
-            if (q < top) { jj = stk_job[q]; ff = stk_fin[q]; live = sst[jj] == ff - O[jj]; }
-            const unsigned m = __ballot_sync(0xffffffffu, live);
-            __syncwarp();
-            if (live) { const int d = w + __popc(m & lt_mask); stk_job[d] = jj; stk_fin[d] = ff; }
-            w += __popc(m);
-            __syncwarp();
+        const bool ok = fr && need <= room;
+        const unsigned okm = __ballot_sync(0xffffffffu, ok);
+        const int m = __popc(okm);
+        if (m) {
+          if (top + 32 > static_cast<int>(cap) || top > 2 * cnt + 64) {   // mostly stale entries: keep the live ones, in order
+            int w = 0;
+            for (int q0 = 0; q0 < top; q0 += 32) {
+              const int qq = q0 + lane;
+              bool live = false;
+              int jj = 0, ff = 0;
+              if (qq < top) { jj = stk_job[qq]; ff = stk_fin[qq]; live = sst[jj] == ff - O[jj]; }
+              const unsigned lm = __ballot_sync(0xffffffffu, live);
+              __syncwarp();
+              if (live) { const int d = w + __popc(lm & lt_mask); stk_job[d] = jj; stk_fin[d] = ff; }
+              w += __popc(lm);
+              __syncwarp();
+            }
+            top = w;
           }
-          top = w;
+          const int fin = ok ? t + O[j] : NEVER;
+          if (ok) {
+            const int d = top + __popc(okm & lt_mask);
+            sst[j] = t; stk_job[d] = j; stk_fin[d] = fin;
+          }
+          __syncwarp();
+          top += m;
+          A += warp_sum(ok ? static_cast<i64>(sj) + 1 - t : static_cast<i64>(0));
+          cnt += m;
+          next_comp = min(next_comp, warp_min_int(fin));
         }
-        __syncwarp();
-        const int fin = t + O[j];
-        if (lane == 0) { sst[j] = t; stk_job[top] = j; stk_fin[top] = fin; }
-        __syncwarp();
-        ++top;
-        A += static_cast<i64>(sc) + 1 - t;
-        ++cnt;
-        next_comp = min(next_comp, fin);
-        ++fpos; cj = -1;
+        const unsigned failed = hit & ~okm;
+        if (failed) {                                   // the first free job that does not fit is the candidate from now on
+          const int src = __ffs(static_cast<int>(failed)) - 1;
+          fpos += src;
+          cj = __shfl_sync(0xffffffffu, j, src);
+          cs = __shfl_sync(0xffffffffu, sj, src);
+          break;
+        }
+        fpos += 32; cj = -1;
       }
       // (5) the round's memory
       const i64 mem = B + A + static_cast<i64>(t) * cnt;
