@@ -561,6 +561,11 @@ def run_fused_workload(args, rank, world, dev, local, dist, binding, Scheduler):
                      "step_frac": stage_bytes / sec_per_step / 1e9 / peak_gbs},
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
     }
+    if n_post:
+        post = "k_refill" if "GBAD" in fams else "k_spec"
+        line["roofline"]["kernel"] = "k_fused_eval<full> + " + post + " (timed together)"
+        line["roofline"]["note"] = (post + " applies a sequential rule per evaluation, one warp each: it is bound by the latency of "
+                                    "dependent loads, and the HBM fraction is given for completeness only")
     if e2e:
         line["e2e"] = {"value": steps_all / (e2e_s / args.steps), "unit": UNIT, "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2],
                        "result": "scalars only (no per-job results and no profile leave the device on this path)"}

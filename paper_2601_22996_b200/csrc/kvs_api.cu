@@ -397,8 +397,9 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     if (ce != cudaSuccess) return fail_cuda(ctx, ce, "refill launch");
   }
   if (do_profile && !spec.empty()) {
-    // the list shares the refill list's region (together at most P entries); the working storage is the fused
-    // kernels' per-CTA scratch, free once they have run
+    // the list shares the refill list's region (together at most P entries); the working storage is everything
+    // the ordering and fused kernels (and the refill) kept between them - the orders, sorted copies, prefix sums
+    // and per-CTA scratch, one contiguous stretch of the workspace - free once they have run
     unsigned char* const list_dev = ws + L.refill_list + refill.size() * 8;
     ce = cudaMemcpyAsync(list_dev, spec.data(), spec.size() * 8, cudaMemcpyHostToDevice, ctx->stream);
     if (ce != cudaSuccess) return fail_cuda(ctx, ce, "copy of the list of speculative evaluations");
@@ -411,8 +412,8 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     q.profile_off = v.profile_off; q.profile = v.profile;
     q.peak = v.peak; q.flow = v.flow; q.horizon = v.horizon; q.job_steps = v.job_steps; q.n_runs = o.n_runs;
     q.n_unfinished = v.n_unfinished; q.feasible = v.feasible; q.status = v.status;
-    q.scratch = ws + L.lists; q.max_jobs = max_n;
-    const i64 room = static_cast<i64>(L.counter - L.lists) / kvs_spec_warp_bytes(max_n);
+    q.scratch = ws + L.perm; q.max_jobs = max_n;
+    const i64 room = static_cast<i64>(L.counter - L.perm) / kvs_spec_warp_bytes(max_n);
     const i64 want = static_cast<i64>(ctx->sm_count) * 32;
     q.n_warps = std::min<i64>(std::min<i64>(room, want), q.n_list);
     q.counter = counters + 24;
