@@ -1,5 +1,6 @@
-"""One full pass per config: EVERY evaluation of configs 2, 3 and 5 (chunk of instances by chunk) and
-EVERY cell of config 4's two sweeps against the oracle, element by element.
+"""One full pass per config: EVERY evaluation of configs 2, 3 and 5 (chunk of instances by chunk), of config 2
+under the dynamic refill and under speculative runs, and EVERY cell of config 4's two sweeps against the oracle,
+element by element.
 
 This takes tens of minutes of host time (the oracle is single-threaded code, run here on all host
 cores over disjoint evaluations), so it is not part of the `-m gpu` suite: it is selected with
@@ -22,7 +23,7 @@ from paper_2601_22996_b200 import binding, workloads
 
 pytestmark = pytest.mark.full
 
-CHUNK = {"c2": 128, "c3": 16, "c5": 256}     # instances per call
+CHUNK = {"c2": 128, "c3": 16, "c5": 256, "c2d": 128, "c2s": 128}     # instances per call
 
 
 def _need():
@@ -90,7 +91,7 @@ def _verify_config(name, pool):
         ctx = sched.context(binding.workspace_bytes(c * n, c, n, P))
         first = Scheduler.scalars(P, dev)
         ctx.build_schedule(inst, settings, dict(n_runs=torch.zeros(P, dtype=torch.int64, device=dev)), first, window=window, max_jobs=n)
-        geo = torch.from_numpy(settings["family"] <= 1).to(dev)
+        geo = torch.from_numpy(np.array([bench.stores_profile(name, int(f)) for f in settings["family"]])).to(dev)
         cap = torch.where(geo, first["horizon"], torch.zeros_like(first["horizon"]))   # as bench.py sizes them
         poff = torch.zeros(P + 1, dtype=torch.int64, device=dev)
         poff[1:] = torch.cumsum(cap, 0)
@@ -135,6 +136,16 @@ def test_full_config3(pool):
 def test_full_config5(pool):
     _need()
     _verify_config("c5", pool)
+
+
+def test_full_config2_dynamic_refill(pool):
+    _need()
+    _verify_config("c2d", pool)
+
+
+def test_full_config2_speculative_runs(pool):
+    _need()
+    _verify_config("c2s", pool)
 
 
 def test_full_config1_and_config4(pool):
