@@ -103,8 +103,9 @@ int kvs_last_timing(kvs_ctx* ctx, float* sort_ms, float* build_ms);
 int kvs_last_timing_split(kvs_ctx* ctx, float* sort_ms, float* light_ms, float* full_ms);
 
 /* Checked build.  A library compiled with -DKVS_DEBUG tests every computed index of the fast fused kernel
- * (shared-memory ring, per-CTA scratch, the caller's profile and per-job outputs) against its bound before
- * the access; a violation is recorded in one device word (code << 56 | index, the first one wins), the
+ * (shared-memory ring, per-CTA scratch, the caller's profile and per-job outputs) and of the refill and
+ * speculative-run kernels (profile rounds, per-job outputs, list, stack and scratch of a warp) against its bound
+ * before the access; a violation is recorded in one device word (code << 56 | index, the first one wins), the
  * access is skipped and the kernel carries on - nothing traps.  This call returns that word for the
  * current device (0 = no violation; synchronises the device) and clears it if `reset` is nonzero;
  * *compiled_in = 1 for a checked build, 0 for a normal one (the word is then always 0).  Either pointer

@@ -412,7 +412,7 @@ int run_fused(kvs_ctx* ctx, const kvs_instances* inst, const kvs_setting* settin
     q.profile_off = v.profile_off; q.profile = v.profile;
     q.peak = v.peak; q.flow = v.flow; q.horizon = v.horizon; q.job_steps = v.job_steps; q.n_runs = o.n_runs;
     q.n_unfinished = v.n_unfinished; q.feasible = v.feasible; q.status = v.status;
-    q.scratch = ws + L.perm; q.max_jobs = max_n;
+    q.scratch = ws + L.perm; q.scratch_bytes = static_cast<i64>(L.counter - L.perm); q.max_jobs = max_n;
     const i64 room = static_cast<i64>(L.counter - L.perm) / kvs_spec_warp_bytes(max_n);
     const i64 want = static_cast<i64>(ctx->sm_count) * 32;
     q.n_warps = std::min<i64>(std::min<i64>(room, want), q.n_list);
@@ -515,6 +515,11 @@ int kvs_debug_check_word(uint64_t* word, int32_t* compiled_in, int32_t reset) {
   int compiled = 0;
   if (cudaDeviceSynchronize() != cudaSuccess) return KVS_E_CUDA;
   if (kvs_fused_check_word(&w, &compiled, reset) != cudaSuccess) return KVS_E_CUDA;
+  // the kernels of the sequential rules keep words of their own: the first violation found is reported
+  unsigned long long w2 = 0ull, w3 = 0ull;
+  if (kvs_refill_check_word(&w2, nullptr, reset) != cudaSuccess || kvs_spec_check_word(&w3, nullptr, reset) != cudaSuccess)
+    return KVS_E_CUDA;
+  if (w == 0ull) w = w2 ? w2 : w3;
   if (word) *word = w;
   if (compiled_in) *compiled_in = compiled;
   return KVS_OK;

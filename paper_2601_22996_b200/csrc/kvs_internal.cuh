@@ -141,6 +141,7 @@ struct SpecParams {
   i64* peak; i64* flow; i64* horizon; i64* job_steps; i64* n_runs; i64* n_unfinished; uint8_t* feasible;
   const int32_t* status;
   unsigned char* scratch;      // n_warps blocks of kvs_spec_warp_bytes(max_jobs) bytes
+  i64 scratch_bytes;
   i64 max_jobs;
   i64 n_warps;                 // warps launched; each takes evaluations from the list until it is used up
   ull* counter;
@@ -167,6 +168,8 @@ enum { KVS_FUSED_ANY = -1 };   // instantiation of the fast kernel for any famil
 cudaError_t kvs_launch_fused(const BuildParams& p, int grid, int light, int fam, cudaStream_t stream);
 int kvs_fused_ctas_per_sm(int light);
 cudaError_t kvs_fused_check_word(unsigned long long* word, int* compiled, int reset);
+cudaError_t kvs_refill_check_word(unsigned long long* word, int* compiled, int reset);
+cudaError_t kvs_spec_check_word(unsigned long long* word, int* compiled, int reset);
 cudaError_t kvs_launch_generic(const GenericParams& p, cudaStream_t stream);
 cudaError_t kvs_launch_refill(const RefillParams& p, cudaStream_t stream);
 i64 kvs_spec_warp_bytes(i64 max_jobs);

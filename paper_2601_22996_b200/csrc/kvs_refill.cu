@@ -11,7 +11,7 @@
 // max over u in [t, t + o) of R(u) <= M - s - 1 + t; if it does not, the maximising round u* rules out every
 // start before min(max R - (M - s - 1), u* + 1), so the search jumps there instead of trying round by round.
 // The plan's array is the caller's profile buffer, which ends up holding the refilled schedule's profile.
-#include "kvs_internal.cuh"
+#include "kvs_check.cuh"
 
 namespace {
 
@@ -32,13 +32,17 @@ __global__ void __launch_bounds__(RT) k_refill(RefillParams p) {
   int32_t* const js = p.job_start + p.job_out_off[e];
   int32_t* const jc = p.job_completion + p.job_out_off[e];
   const i64 H = p.horizon[e];                           // of the batching schedule; within the profile's capacity (status 0)
+  const i64 pcap = p.profile_off[e + 1] - p.profile_off[e];   // bound of every profile index below (checked build)
+  (void)pcap;
   i64 flow = 0;
   int prev = 0, hmax = 0;
   for (int x = 0; x < n; ++x) {
     const int j = p.perm[lo + x];
     const int oj = p.sorted_o[lo + x], sj = p.sorted_s[lo + x];
+    if (!KVS_OK_AT(j, n, CHK_RF_JOB)) continue;
     const int g = js[j];
-    for (int u = lane; u < oj; u += 32) prof[g + u] -= sj + u + 1;
+    for (int u = lane; u < oj; u += 32)
+      if (KVS_OK_AT(g + u, pcap, CHK_RF_PROF_OUT)) prof[g + u] -= sj + u + 1;
     __syncwarp();
     const i64 bound = M - sj - 1;
     int d = g, t = prev;
@@ -47,6 +51,7 @@ __global__ void __launch_bounds__(RT) k_refill(RefillParams p) {
       i64 best = -1;
       int arg = t;
       for (int u = t + lane; u < t + oj; u += 32) {
+        if (!KVS_OK_AT(u, pcap, CHK_RF_PROF_WIN)) continue;
         const i64 r = static_cast<i64>(prof[u]) + u;
         if (r >= best) { best = r; arg = u; }
       }
@@ -60,7 +65,8 @@ __global__ void __launch_bounds__(RT) k_refill(RefillParams p) {
       const i64 need = best - bound;                    // no start before this round clears round `arg`
       t = static_cast<int>(min_i64(need, static_cast<i64>(arg) + 1));
     }
-    for (int u = lane; u < oj; u += 32) prof[d + u] += sj + u + 1;
+    for (int u = lane; u < oj; u += 32)
+      if (KVS_OK_AT(d + u, pcap, CHK_RF_PROF_IN)) prof[d + u] += sj + u + 1;
     __syncwarp();
     if (lane == 0) { js[j] = d; jc[j] = d + oj; }
     flow += d + oj;
@@ -79,6 +85,8 @@ __global__ void __launch_bounds__(RT) k_refill(RefillParams p) {
 }
 
 }  // namespace
+
+KVS_DEFINE_CHECK_WORD(kvs_refill_check_word)
 
 cudaError_t kvs_launch_refill(const RefillParams& p, cudaStream_t stream) {
   if (p.n_list <= 0) return cudaSuccess;

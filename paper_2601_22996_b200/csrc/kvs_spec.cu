@@ -21,6 +21,7 @@
 // it: one over the run starts, one over the slot ends start + tau (nondecreasing in the rank), which is when a
 // killed job becomes free to speculate.  No entry before position `fpos` and none at or after `fhi` is free at the
 // moment; the events that free a job (a slot end, a kill for memory) widen that range, a scan narrows it.
+#include "kvs_check.cuh"
 #include "kvs_ladder.cuh"
 
 namespace {
@@ -66,6 +67,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
   const i64 wslot = static_cast<i64>(blockIdx.x) * SWARPS + warp;
   if (wslot >= p.n_warps) return;
   const i64 cap = p.max_jobs;
+  if (!KVS_OK_AT((wslot + 1) * spec_stride(cap) - 1, p.scratch_bytes, CHK_SP_SCRATCH)) return;
   unsigned char* const mine = p.scratch + wslot * spec_stride(cap);
   int* const pos_of = reinterpret_cast<int*>(mine);    // position of a job in the current phase's list
   int* const sst = pos_of + cap;
@@ -95,6 +97,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
     int32_t* const js = p.job_start + p.job_out_off[e];
     int32_t* const jc = p.job_completion + p.job_out_off[e];
     const int H = static_cast<int>(p.horizon[e]);       // of the slicing schedule; within the profile's capacity (status 0)
+    if (!KVS_OK_AT(H, p.profile_off[e + 1] - p.profile_off[e] + 1, CHK_SP_PROF) || !KVS_OK_AT(n, cap + 1, CHK_SP_JOB)) continue;
     if (n == 0) continue;
 
     // ---- phase table: ladder, classes, participants, first round of every phase ----
@@ -156,7 +159,9 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
             bool fin = false;
             int j = 0, s0 = 0;
             if (f == t) {
-              j = stk_job[q]; s0 = t - O[j];
+              j = stk_job[q];
+              if (!KVS_OK_AT(j, n, CHK_SP_JOB)) j = 0;
+              s0 = t - O[j];
               fin = sst[j] == s0;                       // a live entry
             }
             const unsigned fm = __ballot_sync(0xffffffffu, fin);
@@ -184,7 +189,10 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         for (int r0 = re; r0 < lim; r0 += 32) {
           const int r = r0 + lane;
           bool fr = false;
-          if (r < lim) { const int j = list[r]; fr = !done[j] && sst[j] < 0; }
+          if (r < lim && KVS_OK_AT(r, n, CHK_SP_LIST)) {
+            const int j = list[r];
+            if (KVS_OK_AT(j, n, CHK_SP_JOB)) fr = !done[j] && sst[j] < 0;
+          }
           const unsigned hit = __ballot_sync(0xffffffffu, fr);
           if (hit) { fpos = r0 + __ffs(static_cast<int>(hit)) - 1; cj = -1; break; }
         }
@@ -218,10 +226,11 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         bool cand_started = false;                      // a job that starts may be the known candidate
         for (int r0 = rs; r0 < rend; r0 += 32) {
           const int r = r0 + lane;
-          const bool act = r < rend;
+          bool act = r < rend && KVS_OK_AT(r, n, CHK_SP_LIST);
           int j = 0, oj = 0, sj = 0, s0 = -1;
           bool dn = false;
-          if (act) { j = list[r]; oj = O[j]; sj = S[j]; dn = done[j] != 0; s0 = sst[j]; }
+          if (act) { j = list[r]; act = KVS_OK_AT(j, n, CHK_SP_JOB); }
+          if (act) { oj = O[j]; sj = S[j]; dn = done[j] != 0; s0 = sst[j]; }
           if (cj >= 0 && __ballot_sync(0xffffffffu, act && j == cj)) cand_started = true;
           const int len = oj < static_cast<int>(tau_c) ? oj : static_cast<int>(tau_c);
           const bool run = act && !dn, drop = act && dn;
@@ -254,13 +263,15 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
           unsigned dm = __ballot_sync(0xffffffffu, drop);
           if (dm) {
             if (drop && len <= 64)
-              for (int u = 0; u < len; ++u) atomicSub(&prof[t + u], sj + u + 1);
+              for (int u = 0; u < len; ++u)
+                if (KVS_OK_AT(t + u, H, CHK_SP_DROP)) atomicSub(&prof[t + u], sj + u + 1);
             unsigned lm = __ballot_sync(0xffffffffu, drop && len > 64);
             while (lm) {
               const int src = __ffs(static_cast<int>(lm)) - 1;
               lm &= lm - 1u;
               const int ls = __shfl_sync(0xffffffffu, len, src), ss = __shfl_sync(0xffffffffu, sj, src);
-              for (int u = lane; u < ls; u += 32) atomicSub(&prof[t + u], ss + u + 1);
+              for (int u = lane; u < ls; u += 32)
+                if (KVS_OK_AT(t + u, H, CHK_SP_DROP)) atomicSub(&prof[t + u], ss + u + 1);
             }
             if ((t & 31) != 0) {                        // at a window's first round the window is loaded afterwards
               const int u = lane - (t & 31);            // this lane's round, counted from t
@@ -288,8 +299,9 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         __syncwarp();
         for (int r = re; r < rs; ++r) {
           const int j = list[r];
+          if (!KVS_OK_AT(j, n, CHK_SP_JOB)) continue;
           const int end = jc[j];                        // beyond t only for a completing run of the pipeline in progress
-          if (end > t) {
+          if (end > t && KVS_OK_AT(end, H + 1, CHK_SP_PROF)) {
             const int first = end - O[j], sj = S[j];
             for (int u = t + lane; u < end; u += 32) prof[u] += sj + (u - first) + 1;
             __syncwarp();
@@ -312,6 +324,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         while (top > 0) {                               // the live entry nearest to the top
           --top;
           const int jj = stk_job[top];
+          if (!KVS_OK_AT(jj, n, CHK_SP_JOB)) continue;
           s0 = stk_fin[top] - O[jj];
           if (sst[jj] == s0) { j = jj; break; }
         }
@@ -324,6 +337,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         if (lane == 0) sst[j] = -1;
         __syncwarp();
         const int a = pos_of[j];                        // free again: it may come before the known candidate
+        if (!KVS_OK_AT(a, np, CHK_SP_LIST)) break;
         if (a < fpos) { fpos = a; cj = -1; }
         if (a >= fhi) { fhi = a + 1; if (cj == -2) cj = -1; }
       }
@@ -338,7 +352,10 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
         const int q = fpos + lane;
         bool fr = false;
         int j = 0, sj = 0;
-        if (q < fhi && !(q >= re && q < rs)) { j = list[q]; fr = !done[j] && sst[j] < 0; }
+        if (q < fhi && !(q >= re && q < rs) && KVS_OK_AT(q, n, CHK_SP_LIST)) {
+          j = list[q];
+          if (KVS_OK_AT(j, n, CHK_SP_JOB)) fr = !done[j] && sst[j] < 0; else j = 0;
+        }
         const unsigned hit = __ballot_sync(0xffffffffu, fr);
         if (!hit) { fpos += 32; cj = -1; continue; }
         if (fr) sj = S[j];
@@ -370,7 +387,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
           const int fin = ok ? t + O[j] : NEVER;
           if (ok) {
             const int d = top + __popc(okm & lt_mask);
-            sst[j] = t; stk_job[d] = j; stk_fin[d] = fin;
+            if (KVS_OK_AT(d, cap, CHK_SP_STACK)) { sst[j] = t; stk_job[d] = j; stk_fin[d] = fin; }
           }
           __syncwarp();
           top += m;
@@ -390,7 +407,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
       }
       // (5) the round's memory
       const i64 mem = B + A + static_cast<i64>(t) * cnt;
-      if (lane == 0) prof[t] = static_cast<int32_t>(mem);
+      if (lane == 0 && KVS_OK_AT(t, H, CHK_SP_PROF)) prof[t] = static_cast<int32_t>(mem);
       peak = max_i64(peak, mem);
       if (cnt == 0) top = 0;                            // only stale entries are left
     }
@@ -409,6 +426,8 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
 }
 
 }  // namespace
+
+KVS_DEFINE_CHECK_WORD(kvs_spec_check_word)
 
 i64 kvs_spec_warp_bytes(i64 max_jobs) { return spec_stride(max_jobs); }
 

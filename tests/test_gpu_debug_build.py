@@ -1,5 +1,5 @@
-"""The checked build of the library (-DKVS_DEBUG): every computed index of the fast fused kernel is tested
-against its bound before the access, a violation is recorded in one device word and the access skipped.
+"""The checked build of the library (-DKVS_DEBUG): every computed index of the fast fused kernel and of the
+refill and speculative-run kernels is tested against its bound before the access, a violation is recorded in one device word and the access skipped.
 compute-sanitizer is not available on the GPU pool, so this is the memory-safety evidence: the tiny, edge,
 window and estimate parity cases run against the checked library in a child process (the binding keeps one
 library per process) and must leave the word at 0 while still matching the oracle bit for bit."""
@@ -53,6 +53,16 @@ parity.check_batch(c2, binding.settings_grid(range(3), ["GBA", "GSA", "SPS", "SI
 c5 = workloads.config5(n_inst=4, n=50_000)
 st = binding.settings_grid(range(4), ["GBA", "GSA"], c5.meta["M_per_instance"].numpy()[:, None])
 parity.check_batch(c5, st, want_runs=False, label="checked config 5")
+# the kernels of the two heuristics: hand-sized, ragged and config-2 cases
+heur = workloads.random_small(913, 40, 60, 30, 90)
+rows = []
+for i in range(heur.n_instances):
+    a, b = int(heur.job_off[i]), int(heur.job_off[i + 1])
+    if b > a:
+        M = int(heur.s[a:b].max() + heur.o[a:b].max()) + 11 * i
+        rows += [dict(instance=i, family=f, M=M, alpha=((2, 1), (3, 2))[i % 2]) for f in ("GBAD", "GSAS")]
+parity.check_batch(heur, binding.make_settings(rows), want_runs=False, label="checked heuristics tiny")
+parity.check_batch(c2, binding.settings_grid(range(3), ["GBAD", "GSAS"], [1 << 17, 1 << 20, 1 << 24]), want_runs=False, label="checked heuristics config 2")
 torch.cuda.synchronize()
 word, _ = binding.debug_check_word()
 print("CHECK_WORD", hex(word))
