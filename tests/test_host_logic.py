@@ -31,6 +31,18 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding._SweepParams) == 72 and binding._SweepParams.beta0.offset == 48 and ctypes.sizeof(binding._SweepOut) == 48
 
 
+def test_family_and_status_codes_match_the_header():
+    """The binding and the oracle number the schedule families like `enum kvs_family`; the status bits the tests
+    read are those of `enum kvs_eval_status`."""
+    import oracle
+    header = open(os.path.join(ROOT, "include", "kvs.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    fam = dict((k, int(v)) for k, v in re.findall(r"KVS_(GBA|GSA|SPS|SIMS|GBAD|GSAS)\s*=\s*(\d+)", header))
+    assert fam == binding.FAMILY == oracle.FAMILY and len(fam) == 6
+    bits = dict((k, int(v, 0)) for k, v in re.findall(r"KVS_EVAL_([A-Z_]+)\s*=\s*(0x[0-9a-fA-F]+|\d+)", header))
+    assert bits["INFEASIBLE"] == binding.EVAL_INFEASIBLE and bits["BAD_INPUT"] == binding.EVAL_BAD_INPUT
+
+
 def test_no_gpu_means_a_loud_failure():
     if torch.cuda.is_available():
         pytest.skip("a GPU is present")
