@@ -30,6 +30,7 @@ constexpr int ST = 128;                 // threads per CTA: four warps, one eval
 constexpr int SWARPS = ST / 32;
 constexpr int MAXP = KVS_MAX_PHASES;
 constexpr int NEVER = 0x7fffffff;
+constexpr u32 NO_ROUND = 0xffffffffu;   // completion rounds are kept as 32-bit unsigned: t + o stays below 2^32
 
 struct SpecShared {
   u128 pw_a[MAXP + 1];
@@ -45,7 +46,11 @@ __device__ __forceinline__ i64 slot_of(int r, u32 tau, u32 k) {
   return (x >> 32) == 0 ? static_cast<i64>(static_cast<u32>(x) / k) : static_cast<i64>(x / k);
 }
 
-__device__ __forceinline__ int warp_min_int(int v) { return -warp_max(-v); }
+__device__ __forceinline__ u32 warp_min_u32(u32 v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, d));
+  return v;
+}
 
 // Number of ranks r < np with floor(r * tau / k) <= x: r * tau < (x + 1) * k, so ceil((x + 1) * k / tau) of them.
 __device__ __forceinline__ int started(i64 x, u32 tau, u32 k, int np) {
@@ -135,7 +140,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
     i64 ns = 0, ne = tau_c;                             // their rounds
     i64 A = 0;                                          // speculative runs hold A + t * cnt tokens in round t
     int cnt = 0, top = 0;                               // running speculative runs; entries on the stack (some stale)
-    int next_comp = NEVER;                              // no speculative run completes before this round
+    u32 next_comp = NO_ROUND;                           // no speculative run completes before this round
     int fpos = 0, fhi = n;
     int cj = -1, cs = 0;                                // the free job at fpos and its prompt length, while known (cj = -2: none is free)
     int left = n;
@@ -144,21 +149,22 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
     int Bw = 0;                                         // lane l holds the plan's memory of round (t & ~31) + l
     for (int t = 0; t <= H; ++t) {
       // (1) speculative completions
-      if (t == next_comp) {
-        int nc = NEVER;
+      const u32 tu = static_cast<u32>(t);
+      if (tu == next_comp) {
+        u32 nc = NO_ROUND;
         for (int g0 = 0; g0 < top; g0 += 128) {         // four chunks' completion rounds are loaded together
-          int fq[4];
+          u32 fq[4];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) fq[c] = g0 + 32 * c + lane < top ? stk_fin[g0 + 32 * c + lane] : NEVER;
+          for (int c = 0; c < 4; ++c) fq[c] = g0 + 32 * c + lane < top ? static_cast<u32>(stk_fin[g0 + 32 * c + lane]) : NO_ROUND;
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const int q = g0 + 32 * c + lane;
-            const int f = fq[c];
-            if (f > t) nc = min(nc, f);                 // stale entries included: they cost one empty scan at most
-            if (__ballot_sync(0xffffffffu, f == t) == 0) continue;
+            const u32 f = fq[c];
+            if (f > tu) nc = min(nc, f);                // stale entries included: they cost one empty scan at most
+            if (__ballot_sync(0xffffffffu, f == tu) == 0) continue;
             bool fin = false;
             int j = 0, s0 = 0;
-            if (f == t) {
+            if (f == tu) {
               j = stk_job[q];
               if (!KVS_OK_AT(j, n, CHK_SP_JOB)) j = 0;
               s0 = t - O[j];
@@ -176,7 +182,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
             }
           }
         }
-        next_comp = warp_min_int(nc);
+        next_comp = warp_min_u32(nc);
         __syncwarp();
       }
       // slots that have ended: a job killed at the end of its slot is free again.  The ranks whose slots end by
@@ -325,7 +331,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
           --top;
           const int jj = stk_job[top];
           if (!KVS_OK_AT(jj, n, CHK_SP_JOB)) continue;
-          s0 = stk_fin[top] - O[jj];
+          s0 = static_cast<int>(static_cast<u32>(stk_fin[top]) - static_cast<u32>(O[jj]));
           if (sst[jj] == s0) { j = jj; break; }
         }
         if (j < 0) break;
@@ -375,7 +381,7 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
               const int qq = q0 + lane;
               bool live = false;
               int jj = 0, ff = 0;
-              if (qq < top) { jj = stk_job[qq]; ff = stk_fin[qq]; live = sst[jj] == ff - O[jj]; }
+              if (qq < top) { jj = stk_job[qq]; ff = stk_fin[qq]; live = sst[jj] == static_cast<int>(static_cast<u32>(ff) - static_cast<u32>(O[jj])); }
               const unsigned lm = __ballot_sync(0xffffffffu, live);
               __syncwarp();
               if (live) { const int d = w + __popc(lm & lt_mask); stk_job[d] = jj; stk_fin[d] = ff; }
@@ -384,16 +390,16 @@ __global__ void __launch_bounds__(ST) k_spec(SpecParams p) {
             }
             top = w;
           }
-          const int fin = ok ? t + O[j] : NEVER;
+          const u32 fin = ok ? tu + static_cast<u32>(O[j]) : NO_ROUND;
           if (ok) {
             const int d = top + __popc(okm & lt_mask);
-            if (KVS_OK_AT(d, cap, CHK_SP_STACK)) { sst[j] = t; stk_job[d] = j; stk_fin[d] = fin; }
+            if (KVS_OK_AT(d, cap, CHK_SP_STACK)) { sst[j] = t; stk_job[d] = j; stk_fin[d] = static_cast<int>(fin); }
           }
           __syncwarp();
           top += m;
           A += warp_sum(ok ? static_cast<i64>(sj) + 1 - t : static_cast<i64>(0));
           cnt += m;
-          next_comp = min(next_comp, warp_min_int(fin));
+          next_comp = min(next_comp, warp_min_u32(fin));
         }
         const unsigned failed = hit & ~okm;
         if (failed) {                                   // the first free job that does not fit is the candidate from now on
