@@ -58,7 +58,9 @@ enum kvs_family { KVS_GBA = 0, KVS_GSA = 1, KVS_SPS = 2, KVS_SIMS = 3,
                    * schedule is formed first and kept; round by round, memory it leaves free starts further runs of
                    * jobs that are neither done nor running, lowest index first, as long as the first round of the
                    * next one fits; when the schedule's own runs need the memory the speculative run started last is
-                   * killed; a job completed by a speculative run drops out of the schedule's later phases.  No job
+                   * killed; a job completed by a speculative run drops out of the schedule's later phases.  job_start and
+                   * job_completion are those of the run that completed the job; job_steps and n_runs count every executed
+                   * run, the rounds of killed speculative runs included; the profile holds both kinds of runs.  No job
                    * completes later than in the slicing schedule.  Accepted like KVS_GBAD (job_start, job_completion
                    * and a profile with the slicing schedule's horizon as capacity are the working storage;
                    * kvs_build_schedule reports the slicing schedule); offline instances without estimates, staggered
