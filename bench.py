@@ -561,6 +561,10 @@ def run_fused_workload(args, rank, world, dev, local, dist, binding, Scheduler):
                      "step_frac": stage_bytes / sec_per_step / 1e9 / peak_gbs},
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
     }
+    if traffic is not None and full_avg > 0:
+        # the measured DRAM traffic of the same launches over their duration: what the memory system actually sustained
+        line["roofline"]["dram_gbs"] = traffic / (full_avg * 1e-3) / 1e9
+        line["roofline"]["dram_frac"] = line["roofline"]["dram_gbs"] / peak_gbs
     if n_post:
         post = "k_refill" if "GBAD" in fams else "k_spec"
         line["roofline"]["kernel"] = "k_fused_eval<full> + " + post + " (timed together)"
