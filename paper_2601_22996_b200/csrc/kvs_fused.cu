@@ -1250,16 +1250,18 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
         } else {
           // Z[m] = sum over ranks j < m of (s_j - start_j): the jobs [i, b) active in round t hold
           // Z[b] - Z[i] + (b - i)(t + 1) tokens.  First Z for every rank, then one candidate per run.
+          // four ranks per thread and step: shorter dependent chains than the ring's rounds per thread
+          constexpr int EVI = 4;
           u32* const Z = reinterpret_cast<u32*>(cls);      // N + 1 words of this CTA's scratch
           const u32 qt = tau / k, rt = tau - qt * k;
           u32 F_run = 0;
-          for (u32 c0 = 0; c0 <= N; c0 += TILE) {
-            const u32 r = c0 + ITEMS * tid;
+          for (u32 c0 = 0; c0 <= N; c0 += (T * EVI)) {
+            const u32 r = c0 + EVI * tid;
             u32 q = 0, rem = 0;
             if (r <= N) { u64 dq_, dr_; divmod_u(static_cast<u64>(r) * tau, k, &dq_, &dr_); q = static_cast<u32>(dq_); rem = static_cast<u32>(dr_); }
-            u32 f[ITEMS], tot = 0;
+            u32 f[EVI], tot = 0;
 #pragma unroll
-            for (int j = 0; j < ITEMS; ++j) {
+            for (int j = 0; j < EVI; ++j) {
               f[j] = tot;
               if (r + j < N) tot += q;
               rem += rt; q += qt;
@@ -1284,24 +1286,24 @@ __global__ void __launch_bounds__(KVS_EVAL_THREADS, LIGHT ? KVS_EVAL_MIN_CTAS + 
             const u32 off = F_run + __shfl_sync(0xffffffffu, wi - w, warp) + (incl - tot);
             F_run += __shfl_sync(0xffffffffu, wi, 31);
 #pragma unroll
-            for (int j = 0; j < ITEMS; ++j)
+            for (int j = 0; j < EVI; ++j)
               if (r + j <= N && KVS_IN(r + j, z_cap, CHK_Z)) Z[r + j] = ps32[2 * static_cast<size_t>(r + j)] - (off + f[j]);
           }
           __syncthreads();
-          for (u32 c0 = 0; c0 < N; c0 += TILE) {
-            const u32 r = c0 + ITEMS * tid;
+          for (u32 c0 = 0; c0 < N; c0 += (T * EVI)) {
+            const u32 r = c0 + EVI * tid;
             if (r >= N) continue;
             u64 dq_, dr_;
             divmod_u(static_cast<u64>(r) * tau, k, &dq_, &dr_);
             u32 q = static_cast<u32>(dq_), rem = static_cast<u32>(dr_);
-            u32 o_[ITEMS], z_[ITEMS];
+            u32 o_[EVI], z_[EVI];
 #pragma unroll
-            for (int j = 0; j < ITEMS; ++j) {
+            for (int j = 0; j < EVI; ++j) {
               o_[j] = r + j < N ? static_cast<u32>(__ldg(Ow + r + j)) : 0u;
               z_[j] = (r + j < N && KVS_IN(r + j, z_cap, CHK_Z)) ? Z[r + j] : 0u;
             }
 #pragma unroll
-            for (int j = 0; j < ITEMS; ++j) {
+            for (int j = 0; j < EVI; ++j) {
               if (r + j < N) {
                 const u32 t1 = q + min(o_[j], tau);                       // last round of the run, plus one
                 const u64 x = static_cast<u64>(t1) * k + (tau - 1u);      // b = ranks that start before t1
